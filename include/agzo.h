@@ -1,0 +1,208 @@
+/*
+ * agzo.h -- C ABI of the B200 (sm_100a) implementation of the per-step hot path of AGZO,
+ * Activation-Guided Zeroth-Order optimisation.
+ *
+ * For every linear layer l with weight W_l (d_out x d_in) and the input activations of
+ * the current minibatch H_l (d_in x m, given here as X = H^T, one token per row):
+ *   1. Algorithm 1 (SubspaceExtract): an orthonormal basis A_l (d_in x r) of a rank-r
+ *      subspace of col(H_l) by K steps of block power iteration from a Gaussian test
+ *      matrix.  Stored as V = A^T: r rows of length d_in.
+ *   2. Eq. (agzo-perturb): Delta_l = R_l A_l^T with R_l (d_out x r) i.i.d. N(0,1),
+ *      regenerated from a counter-based seed every time it is needed; the d_out x d_in
+ *      matrix Delta_l is never stored.
+ *   3. Algorithm 2: W <- W + mu*Delta in place, loss, (two-point mode: W <- W - 2mu*Delta,
+ *      loss,) the projected-gradient scalar g, and the fused restore-and-update pass.
+ *
+ * Conventions shared by all calls
+ *   - Every data pointer is a DEVICE pointer unless its name starts with "h_" or the text
+ *     says "host".  Layer descriptor arrays are HOST arrays, read during the call only.
+ *   - W is [d_out][ldw] row-major (the layout of a torch nn.Linear weight), bf16 or fp32.
+ *     X is [m][ldx] row-major, bf16 or fp32.  V is [r][ldv] row-major fp32, ldv >= d_in.
+ *   - The library allocates no device memory.  Scratch comes from the workspace handed to
+ *     agzo_create; it must stay valid and must not be touched by the caller while a call
+ *     that uses it is in flight.  The library keeps no other pointer past a call.
+ *   - All work is enqueued on the caller's stream (a cudaStream_t passed as void*) and the
+ *     calls return without waiting for it, except where stated.  Calls that share a context
+ *     must be issued on one stream or be ordered by the caller.
+ *   - Every function returns an agzo_status; nothing throws, traps or aborts.  Argument
+ *     errors are detected on the host before anything is launched.  Conditions that only
+ *     the device can see (a rank-deficient panel, a wait that ran out) are written to a
+ *     status word in the workspace and reported by agzo_poll.
+ *   - Random streams: Philox4x32-10 with key = the 64-bit step seed and counter
+ *     (b_lo, b_hi, layer_id, tag); b = e >> 2 where e is the row-major index of the element
+ *     inside the matrix being drawn, which takes output word e & 3 of that block.
+ *     tag 0 = R_l (d_out x r), tag 1 = Omega (m x r), tag 2 = dense direction.
+ *     Normals are Box-Muller on the word pairs (x0,x1) and (x2,x3):
+ *       u1 = ((x >> 8) + 1) * 2^-24, u2 = (x' >> 8) * 2^-24, s = sqrt(-2 ln u1),
+ *       even lane = s*cos(2 pi u2), odd lane = s*sin(2 pi u2), in fp32.
+ */
+#ifndef AGZO_H_
+#define AGZO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct agzo_ctx agzo_ctx;
+
+typedef enum agzo_status {
+  AGZO_OK = 0,
+  AGZO_ERR_INVALID_ARG = 1,   /* null pointer, bad size, bad alignment, r out of range      */
+  AGZO_ERR_UNSUPPORTED = 2,   /* a dtype / mode combination the library does not implement  */
+  AGZO_ERR_CUDA = 3,          /* a CUDA runtime call failed; agzo_last_cuda_error has the code */
+  AGZO_ERR_WORKSPACE = 4,     /* workspace missing, misaligned or too small for these layers */
+  AGZO_ERR_STATE = 5,         /* call made on a destroyed / foreign context                 */
+  AGZO_ERR_TIMEOUT = 6,       /* a bounded device-side wait ran out (reported by agzo_poll)  */
+  AGZO_ERR_CALLBACK = 7,      /* the loss callback of agzo_step returned non-zero           */
+  AGZO_WARN_RANK_DEFICIENT = 100 /* some panel had a column with R_kk <= 1e-4 R_11; that
+                                    column of V is zero (reported by agzo_poll)             */
+} agzo_status;
+
+typedef enum agzo_dtype { AGZO_BF16 = 0, AGZO_F32 = 1 } agzo_dtype;
+
+#define AGZO_MAX_RANK 64
+#define AGZO_MAX_LAYERS 4096
+
+/* One linear layer.  Plain data, no ownership.  Fields a call does not use may be NULL/0:
+ * the in-place passes ignore X, ldx, x_dtype, m; extraction ignores W, W16.               */
+typedef struct agzo_layer {
+  void*       W;        /* [d_out][ldw], w_dtype; perturbed and updated in place           */
+  int64_t     ldw;      /* row pitch of W in elements, >= d_in                             */
+  void*       W16;      /* optional bf16 compute copy of an fp32 master W, else NULL.  When
+                           present, W is never perturbed: perturb writes
+                           W16 = bf16(W + c*Delta), update writes W += c*Delta; W16 = bf16(W) */
+  int64_t     ldw16;
+  const void* X;        /* [m][ldx], x_dtype: H_l^T, read only by extraction               */
+  int64_t     ldx;
+  float*      V;        /* [r][ldv] fp32: A_l^T, written by extraction, read by the passes */
+  int64_t     ldv;
+  int32_t     w_dtype;  /* agzo_dtype of W                                                 */
+  int32_t     x_dtype;  /* agzo_dtype of X                                                 */
+  int32_t     d_out;
+  int32_t     d_in;
+  int32_t     m;        /* tokens (b*T of Section 3.1)                                     */
+  int32_t     r;        /* 1 <= r <= min(AGZO_MAX_RANK, d_in, m)                           */
+  uint32_t    layer_id; /* enters the Philox counter: the per-layer seed s_l of Algorithm 2 */
+  uint32_t    reserved; /* must be 0                                                       */
+} agzo_layer;
+
+typedef struct agzo_params {
+  uint64_t seed;  /* step seed (Philox key)                                                */
+  float    eps;   /* smoothing parameter mu                                                */
+  float    lr;    /* step size eta                                                         */
+  int32_t  K;     /* power-iteration steps of Algorithm 1 (the paper uses 3), 0 <= K <= 16 */
+  int32_t  mode;  /* 0: two-point g = (f+ - f-)/(2 mu); 1: Algorithm 2 as printed,
+                     g = (f+ - f0)/mu                                                      */
+} agzo_params;
+
+/* Loss callback of agzo_step: run the model's forward on `stream` with the weights as they
+ * are now and leave the scalar loss (fp32) at d_loss (device).  phase: 0 = unperturbed
+ * forward, during or after which the X buffers of the descriptors must have been filled
+ * (Algorithm 2, step 1), 1 = at W + mu*Delta, 2 = at W - mu*Delta.  Return 0 on success. */
+typedef int (*agzo_loss_fn)(void* user, void* stream, int phase, float* d_loss);
+
+/* ---------------------------------------------------------------- context and workspace */
+
+/* Bytes of workspace that every call on these layers needs (host only, no CUDA call).
+ * A workspace sized for one layer list is also valid for any list whose per-field maxima
+ * and layer count are not larger.  Error: INVALID_ARG for a bad descriptor.              */
+agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_bytes);
+
+/* Creates a context bound to CUDA device `device` that will use `workspace`
+ * (device memory, 256-byte aligned, workspace_bytes long; owned by the caller, who frees
+ * it after agzo_destroy).  Synchronous: it clears the device status word.                */
+agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t workspace_bytes);
+agzo_status agzo_destroy(agzo_ctx* ctx);
+
+/* Options: "extract_path" 0 = automatic, 1 = CUDA-core fp32 kernels only, 2 = require the
+ * tensor-core kernels (UNSUPPORTED at call time if a layer cannot use them);
+ * "wave_bytes" = activation bytes grouped into one launch wave of extraction.            */
+agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value);
+
+/* Waits for the stream work of this context issued so far on `stream` and returns the
+ * device status word: AGZO_OK, AGZO_WARN_RANK_DEFICIENT or AGZO_ERR_TIMEOUT; the word is
+ * cleared.  The only synchronising call besides create.                                  */
+agzo_status agzo_poll(agzo_ctx* ctx, void* stream);
+
+const char* agzo_status_string(agzo_status s);
+int         agzo_last_cuda_error(const agzo_ctx* ctx);
+
+/* ---------------------------------------------------------------- Algorithm 1 */
+
+/* SubspaceExtract(H_l, r_l, K) for every layer: Omega_l (m x r) Gaussian from
+ * (seed, layer_id, tag 1); Y = H Omega; K times { Q = qr(Y); Y = H (H^T Q) }; A = qr(Y).Q.
+ * qr is the unique thin factorisation with a positive diagonal.  Writes V = A^T.
+ * X may be released as soon as the stream work of this call has completed.
+ * Errors: INVALID_ARG (null X or V, r > min(d_in, m), ldv < d_in, K out of range),
+ * WORKSPACE.  Rank-deficient panels are reported through agzo_poll.                      */
+agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int n,
+                                  uint64_t seed, int K, void* stream);
+
+/* ---------------------------------------------------------------- Eq. (agzo-perturb), Algorithm 2 */
+
+/* W_l <- W_l + scale * R_l A_l^T for every layer, R_l regenerated from (seed, layer_id,
+ * tag 0): step 2 of Algorithm 2 with scale = mu; the two-point flip is scale = -2 mu.
+ * One fused read-modify-write pass; fp32 arithmetic, one rounding to the storage type.
+ * With a W16 compute copy: W16 <- bf16(W + scale * Delta), W untouched.                   */
+agzo_status agzo_perturb(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                         float scale, void* stream);
+
+/* W_l <- W_l - scale * R_l A_l^T: the "restore" half of step 3 of Algorithm 2.  It is the
+ * same pass as agzo_perturb with the opposite sign, not a bit-exact undo: in bf16 storage
+ * mu*Delta can be below one ulp of W.  With a W16 copy: W16 <- bf16(W).                   */
+agzo_status agzo_restore(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                         float scale, void* stream);
+
+/* W_l <- W_l - lr * g * R_l A_l^T with g read from device memory (d_ghat): the "update"
+ * half of step 3.  With a W16 copy the master is updated and W16 <- bf16(W).             */
+agzo_status agzo_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                        float lr, const float* d_ghat, void* stream);
+
+/* The projected-gradient scalar (Algorithm 2, step 3; Eq. agzo-estimator), on the device:
+ * mode 0: *d_ghat = (*d_f_plus - *d_f_other) / (2 eps)   (f_other = f at W - eps*Delta)
+ * mode 1: *d_ghat = (*d_f_plus - *d_f_other) / eps       (f_other = f0)
+ * evaluated in double and rounded to fp32.                                               */
+agzo_status agzo_ghat(agzo_ctx* ctx, const float* d_f_plus, const float* d_f_other,
+                      float eps, int mode, float* d_ghat, void* stream);
+
+/* Step 3 of Algorithm 2 as one pass: W_l <- W_l + c * R_l A_l^T with
+ * mode 0: c = eps - lr*g (the weights sit at W - eps*Delta after the second forward),
+ * mode 1: c = -(eps + lr*g) (the weights sit at W + eps*Delta), g read from d_ghat,
+ * c formed in double and rounded to fp32.  With a W16 copy: W <- W - lr*g*Delta and
+ * W16 <- bf16(W).                                                                        */
+agzo_status agzo_restore_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n,
+                                uint64_t seed, float eps, float lr, int mode,
+                                const float* d_ghat, void* stream);
+
+/* One AGZO iteration (Algorithm 2): loss(phase 0) -> extract -> perturb(+eps) ->
+ * loss(phase 1) -> [mode 0: perturb(-2 eps) -> loss(phase 2)] -> ghat -> restore_update.
+ * d_out3 (device, 3 floats) receives f_plus, f_other (f_minus or f0) and g.  If the
+ * callback fails, the outstanding perturbation is removed before ERR_CALLBACK returns.   */
+agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n,
+                      const agzo_params* h_params, agzo_loss_fn loss, void* user,
+                      float* d_out3, void* stream);
+
+/* Second case of Eq. (agzo-perturb), for parameters that are not matrices of a linear
+ * layer: w <- w + scale * u with u ~ N(0, I) from (seed, layer_id, tag 2), n_elems
+ * contiguous elements of `dtype`.  If d_scale is not NULL the coefficient is
+ * scale * (*d_scale) (so that the update can use the device-side g).                     */
+agzo_status agzo_perturb_dense(agzo_ctx* ctx, void* w, int64_t n_elems, int dtype,
+                               uint64_t seed, uint32_t layer_id, float scale,
+                               const float* d_scale, void* stream);
+
+/* ---------------------------------------------------------------- test exports */
+
+/* Raw Philox words / normals of elements first .. first+n-1 of stream (seed, layer_id, tag)
+ * written to device memory; used to check the generator bit for bit.                     */
+agzo_status agzo_debug_philox(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, uint32_t tag,
+                              uint64_t first, uint64_t n, uint32_t* d_words, void* stream);
+agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, uint32_t tag,
+                                uint64_t first, uint64_t n, float* d_vals, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AGZO_H_ */

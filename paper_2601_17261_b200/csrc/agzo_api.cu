@@ -1,0 +1,588 @@
+// C ABI of the AGZO library: context, host-side validation, workspace planning and the
+// sequencing of Algorithm 1 / Algorithm 2 over the grouped kernels.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "agzo_common.cuh"
+#include "agzo_tc.cuh"
+
+using namespace agzo;
+
+namespace {
+
+constexpr uint32_t kMagic = 0xA620B200u;
+constexpr size_t kAlign = 256;
+constexpr size_t kHeaderBytes = 256;          // DevStatus + scalar slots
+constexpr size_t kCoefOffset = 64;            // float coefficient slot inside the header
+constexpr int64_t kDefaultWaveBytes = 48ll << 20;
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+struct Plan {
+  std::vector<DevLayer> dev;       // one per layer, scratch pointers filled
+  std::vector<int> tile_start;     // n + 1
+  std::vector<int> wave_end;       // exclusive end index of each extraction wave
+  int total_tiles = 0;
+  int max_r = 0;
+  int fast_mode_mask = 0;          // storage modes present among layers on the vector path
+  bool any_slow = false;           // some layer needs the scalar kernel
+  bool has_extract = false;
+};
+
+}  // namespace
+
+struct agzo_ctx {
+  uint32_t magic;
+  int device;
+  int sm_count;
+  char* ws;
+  size_t ws_bytes;
+  int last_cuda;
+  int extract_path;        // 0 auto, 1 CUDA-core only, 2 tensor-core required
+  int64_t wave_bytes;
+  // descriptors last uploaded
+  std::vector<agzo_layer> cached;
+  bool cached_valid;
+  Plan plan;
+  // pinned staging for the upload
+  void* h_stage;
+  size_t h_stage_bytes;
+  cudaEvent_t stage_ev;
+  bool stage_pending;
+  TcState tc;
+};
+
+namespace {
+
+#define CU(ctx, expr)                              \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) {                      \
+      (ctx)->last_cuda = (int)e__;                 \
+      return AGZO_ERR_CUDA;                        \
+    }                                              \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+enum Need { NEED_RMW = 1, NEED_EXTRACT = 2 };
+
+agzo_status validate(const agzo_layer* L, int n, int need) {
+  if (n < 0 || n > AGZO_MAX_LAYERS) return AGZO_ERR_INVALID_ARG;
+  if (n > 0 && !L) return AGZO_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    const agzo_layer& a = L[i];
+    if (a.reserved != 0) return AGZO_ERR_INVALID_ARG;
+    if (a.d_in < 1 || a.d_out < 0) return AGZO_ERR_INVALID_ARG;
+    if (a.r < 1 || a.r > AGZO_MAX_RANK || a.r > a.d_in) return AGZO_ERR_INVALID_ARG;
+    if (!a.V || a.ldv < a.d_in || (reinterpret_cast<uintptr_t>(a.V) & 3u)) return AGZO_ERR_INVALID_ARG;
+    if (need & NEED_RMW) {
+      if (a.d_out < 1) return AGZO_ERR_INVALID_ARG;
+      if (a.w_dtype != AGZO_BF16 && a.w_dtype != AGZO_F32) return AGZO_ERR_UNSUPPORTED;
+      if (!a.W || a.ldw < a.d_in) return AGZO_ERR_INVALID_ARG;
+      const size_t es = a.w_dtype == AGZO_BF16 ? 2 : 4;
+      if (reinterpret_cast<uintptr_t>(a.W) & (es - 1)) return AGZO_ERR_INVALID_ARG;
+      if (a.W16) {
+        if (a.w_dtype != AGZO_F32) return AGZO_ERR_UNSUPPORTED;
+        if (a.ldw16 < a.d_in || (reinterpret_cast<uintptr_t>(a.W16) & 1u)) return AGZO_ERR_INVALID_ARG;
+      }
+    }
+    if (need & NEED_EXTRACT) {
+      if (a.x_dtype != AGZO_BF16 && a.x_dtype != AGZO_F32) return AGZO_ERR_UNSUPPORTED;
+      if (!a.X || a.m < 1 || a.ldx < a.d_in || a.r > a.m) return AGZO_ERR_INVALID_ARG;
+      const size_t es = a.x_dtype == AGZO_BF16 ? 2 : 4;
+      if (reinterpret_cast<uintptr_t>(a.X) & (es - 1)) return AGZO_ERR_INVALID_ARG;
+    }
+  }
+  return AGZO_OK;
+}
+
+bool has_x(const agzo_layer& a) { return a.X != nullptr && a.m >= 1; }
+
+void slab_shape(const agzo_layer& a, int* slabs, int* slab_rows) {
+  int rows = (a.m + 31) / 32;
+  rows = (rows + 31) / 32 * 32;
+  if (rows < 256) rows = 256;
+  *slab_rows = rows;
+  *slabs = (a.m + rows - 1) / rows;
+}
+
+// scratch bytes one layer needs for extraction (0 when it has no X)
+size_t layer_scratch(const agzo_layer& a, bool tc) {
+  if (!has_x(a)) return 0;
+  int slabs, slab_rows;
+  slab_shape(a, &slabs, &slab_rows);
+  const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
+  const size_t gch = (d + 127) / 128;
+  size_t b = 0;
+  b += align_up(m * r * 4);                 // T
+  b += align_up((size_t)slabs * r * d * 4); // Ypart
+  b += align_up(r * d * 4);                 // Y
+  b += align_up(gch * r * r * 8);           // Gpart
+  b += align_up(r * r * 8);                 // M
+  if (tc) b += tc_layer_scratch(a);
+  return b;
+}
+
+size_t table_bytes(int n) {
+  return align_up((size_t)n * sizeof(DevLayer)) + align_up((size_t)(n + 1) * sizeof(int));
+}
+
+// Builds the device records.  ws == nullptr: only sizes are computed (scratch_needed).
+agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, int64_t wave_bytes,
+                       int extract_path, Plan* plan, size_t* scratch_needed) {
+  plan->dev.assign(n, DevLayer{});
+  plan->tile_start.assign(n + 1, 0);
+  plan->wave_end.clear();
+  plan->max_r = 0;
+  plan->fast_mode_mask = 0;
+  plan->any_slow = false;
+  plan->has_extract = false;
+  const size_t base = kHeaderBytes + table_bytes(n);
+  const size_t scratch_cap = ws ? (ws_bytes > base ? ws_bytes - base : 0) : (size_t)-1;
+  size_t max_wave_scratch = 0;
+
+  int tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const agzo_layer& a = L[i];
+    DevLayer& D = plan->dev[i];
+    D.W = a.W; D.W16 = a.W16; D.X = a.X; D.V = a.V;
+    D.ldw = a.ldw; D.ldw16 = a.ldw16; D.ldx = a.ldx; D.ldv = a.ldv;
+    D.w_dtype = a.w_dtype; D.x_dtype = a.x_dtype;
+    D.d_out = a.d_out; D.d_in = a.d_in; D.m = a.m; D.r = a.r;
+    D.layer_id = a.layer_id;
+    D.rmw_mode = a.W16 ? RMW_PAIR_COMPUTE : (a.w_dtype == AGZO_BF16 ? RMW_BF16 : RMW_F32);
+    const size_t es = a.w_dtype == AGZO_BF16 ? 2 : 4;
+    bool vec = a.W && aligned16(a.W) && (a.ldw * es) % 16 == 0 && a.d_in % 8 == 0 &&
+               aligned16(a.V) && a.ldv % 4 == 0;
+    if (a.W16) vec = vec && aligned16(a.W16) && (a.ldw16 * 2) % 16 == 0;
+    D.vec_ok = vec ? 1 : 0;
+    if (a.W) {
+      if (vec) plan->fast_mode_mask |= 1 << D.rmw_mode; else plan->any_slow = true;
+    }
+    D.tile0 = tiles;
+    D.tiles_c = (a.d_in + 511) / 512;
+    D.tiles_r = a.W ? (a.d_out + 255) / 256 : 0;
+    plan->tile_start[i] = tiles;
+    const long long nt = (long long)D.tiles_c * D.tiles_r;
+    if (tiles + nt > 0x7fffffff) return AGZO_ERR_INVALID_ARG;
+    tiles += (int)nt;
+    if (a.r > plan->max_r) plan->max_r = a.r;
+  }
+  plan->tile_start[n] = tiles;
+  plan->total_tiles = tiles;
+
+  // extraction waves: consecutive layers whose activations fit the wave budget and whose
+  // scratch fits the workspace
+  int i = 0;
+  while (i < n) {
+    if (!has_x(L[i])) { ++i; plan->wave_end.push_back(i); continue; }
+    plan->has_extract = true;
+    size_t used = 0;
+    int64_t xbytes = 0;
+    int j = i;
+    while (j < n && has_x(L[j])) {
+      const bool tc = extract_path != 1 && tc_eligible(L[j]);
+      const size_t need = layer_scratch(L[j], tc);
+      const int64_t xb = (int64_t)L[j].m * L[j].d_in * (L[j].x_dtype == AGZO_BF16 ? 2 : 4);
+      if (j > i && (used + need > scratch_cap || xbytes + xb > wave_bytes)) break;
+      if (used + need > scratch_cap) return AGZO_ERR_WORKSPACE;
+      // carve
+      if (ws) {
+        char* p = ws + base + used;
+        DevLayer& D = plan->dev[j];
+        const agzo_layer& a = L[j];
+        int slabs, slab_rows;
+        slab_shape(a, &slabs, &slab_rows);
+        const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
+        const size_t gch = (d + 127) / 128;
+        D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
+        D.T = reinterpret_cast<float*>(p);      p += align_up(m * r * 4);
+        D.Ypart = reinterpret_cast<float*>(p);  p += align_up((size_t)slabs * r * d * 4);
+        D.Y = reinterpret_cast<float*>(p);      p += align_up(r * d * 4);
+        D.Gpart = reinterpret_cast<double*>(p); p += align_up(gch * r * r * 8);
+        D.M = reinterpret_cast<double*>(p);     p += align_up(r * r * 8);
+        if (tc) tc_carve(a, &D, p);
+      }
+      used += need;
+      xbytes += xb;
+      ++j;
+    }
+    if (used > max_wave_scratch) max_wave_scratch = used;
+    plan->wave_end.push_back(j);
+    i = j;
+  }
+  if (scratch_needed) *scratch_needed = max_wave_scratch;
+  return AGZO_OK;
+}
+
+bool same_layers(const agzo_ctx* c, const agzo_layer* L, int n) {
+  return c->cached_valid && (int)c->cached.size() == n &&
+         (n == 0 || std::memcmp(c->cached.data(), L, (size_t)n * sizeof(agzo_layer)) == 0);
+}
+
+DevLayer* dev_layers(agzo_ctx* c) { return reinterpret_cast<DevLayer*>(c->ws + kHeaderBytes); }
+int* dev_tiles(agzo_ctx* c, int n) {
+  return reinterpret_cast<int*>(c->ws + kHeaderBytes + align_up((size_t)n * sizeof(DevLayer)));
+}
+DevStatus* dev_status(agzo_ctx* c) { return reinterpret_cast<DevStatus*>(c->ws); }
+float* dev_coef(agzo_ctx* c) { return reinterpret_cast<float*>(c->ws + kCoefOffset); }
+
+// Makes the device tables describe `L`; uploads only when the descriptors changed.
+agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
+  if (same_layers(c, L, n)) return AGZO_OK;
+  if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
+  Plan plan;
+  agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, c->wave_bytes, c->extract_path, &plan, nullptr);
+  if (st != AGZO_OK) return st;
+  const size_t lb = align_up((size_t)n * sizeof(DevLayer));
+  const size_t tb = (size_t)(n + 1) * sizeof(int);
+  if (c->stage_pending) {
+    CU(c, cudaEventSynchronize(c->stage_ev));
+    c->stage_pending = false;
+  }
+  if (lb + tb > c->h_stage_bytes) {
+    if (c->h_stage) CU(c, cudaFreeHost(c->h_stage));
+    c->h_stage = nullptr;
+    c->h_stage_bytes = 0;
+    CU(c, cudaMallocHost(&c->h_stage, (lb + tb) * 2));
+    c->h_stage_bytes = (lb + tb) * 2;
+  }
+  if (n > 0) {
+    std::memcpy(c->h_stage, plan.dev.data(), (size_t)n * sizeof(DevLayer));
+    std::memcpy(static_cast<char*>(c->h_stage) + lb, plan.tile_start.data(), tb);
+    CU(c, cudaMemcpyAsync(c->ws + kHeaderBytes, c->h_stage, lb + tb, cudaMemcpyHostToDevice, s));
+    CU(c, cudaEventRecord(c->stage_ev, s));
+    c->stage_pending = true;
+  }
+  c->plan = std::move(plan);
+  c->cached.assign(L, L + n);
+  c->cached_valid = true;
+  return AGZO_OK;
+}
+
+agzo_status check_ctx(agzo_ctx* c) {
+  if (!c || c->magic != kMagic) return AGZO_ERR_STATE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != c->device) {
+    if (cudaSetDevice(c->device) != cudaSuccess) return AGZO_ERR_CUDA;
+  }
+  return AGZO_OK;
+}
+
+agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, float coef,
+                     const float* d_coef, bool pair_update, cudaStream_t s) {
+  agzo_status st = validate(L, n, NEED_RMW);
+  if (st != AGZO_OK) return st;
+  if (n == 0) return AGZO_OK;
+  st = prepare(c, L, n, s);
+  if (st != AGZO_OK) return st;
+  CU(c, launch_rmw(dev_layers(c), dev_tiles(c, n), n, c->plan.total_tiles, c->plan.max_r,
+                   c->plan.fast_mode_mask, c->plan.any_slow, seed, coef, d_coef, pair_update,
+                   c->sm_count, s));
+  return AGZO_OK;
+}
+
+}  // namespace
+
+// =================================================================== C ABI
+extern "C" {
+
+const char* agzo_status_string(agzo_status s) {
+  switch (s) {
+    case AGZO_OK: return "ok";
+    case AGZO_ERR_INVALID_ARG: return "invalid argument";
+    case AGZO_ERR_UNSUPPORTED: return "unsupported dtype or mode";
+    case AGZO_ERR_CUDA: return "CUDA runtime error";
+    case AGZO_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case AGZO_ERR_STATE: return "invalid context";
+    case AGZO_ERR_TIMEOUT: return "device-side wait ran out";
+    case AGZO_ERR_CALLBACK: return "loss callback failed";
+    case AGZO_WARN_RANK_DEFICIENT: return "rank-deficient activation panel";
+  }
+  return "unknown status";
+}
+
+int agzo_last_cuda_error(const agzo_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_bytes) {
+  if (!h_bytes) return AGZO_ERR_INVALID_ARG;
+  agzo_status st = validate(h_layers, n, 0);
+  if (st != AGZO_OK) return st;
+  Plan plan;
+  size_t scratch = 0;
+  st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 0, &plan, &scratch);
+  if (st != AGZO_OK) return st;
+  *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
+  return AGZO_OK;
+}
+
+agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t workspace_bytes) {
+  if (!out) return AGZO_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) ||
+      workspace_bytes < kHeaderBytes)
+    return AGZO_ERR_WORKSPACE;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count)
+    return AGZO_ERR_CUDA;
+  agzo_ctx* c = new (std::nothrow) agzo_ctx();
+  if (!c) return AGZO_ERR_INVALID_ARG;
+  c->magic = kMagic;
+  c->device = device;
+  c->ws = static_cast<char*>(workspace);
+  c->ws_bytes = workspace_bytes;
+  c->last_cuda = 0;
+  c->extract_path = 0;
+  c->wave_bytes = kDefaultWaveBytes;
+  c->cached_valid = false;
+  c->h_stage = nullptr;
+  c->h_stage_bytes = 0;
+  c->stage_pending = false;
+  c->stage_ev = nullptr;
+  cudaError_t e = cudaSetDevice(device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->stage_ev, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaMemset(c->ws, 0, kHeaderBytes);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = tc_init(&c->tc, device);
+  if (e != cudaSuccess) {
+    if (c->stage_ev) cudaEventDestroy(c->stage_ev);
+    delete c;
+    return AGZO_ERR_CUDA;
+  }
+  *out = c;
+  return AGZO_OK;
+}
+
+agzo_status agzo_destroy(agzo_ctx* ctx) {
+  if (!ctx || ctx->magic != kMagic) return AGZO_ERR_STATE;
+  if (ctx->stage_pending) cudaEventSynchronize(ctx->stage_ev);
+  if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+  if (ctx->stage_ev) cudaEventDestroy(ctx->stage_ev);
+  ctx->magic = 0;
+  delete ctx;
+  return AGZO_OK;
+}
+
+agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
+  if (!ctx || ctx->magic != kMagic) return AGZO_ERR_STATE;
+  if (!name) return AGZO_ERR_INVALID_ARG;
+  if (std::strcmp(name, "extract_path") == 0) {
+    if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
+    ctx->extract_path = (int)value;
+  } else if (std::strcmp(name, "wave_bytes") == 0) {
+    if (value < 0) return AGZO_ERR_INVALID_ARG;
+    ctx->wave_bytes = value;
+  } else {
+    return AGZO_ERR_INVALID_ARG;
+  }
+  ctx->cached_valid = false;   // the plan depends on the options
+  return AGZO_OK;
+}
+
+agzo_status agzo_poll(agzo_ctx* ctx, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  DevStatus h{};
+  CU(ctx, cudaMemcpyAsync(&h, dev_status(ctx), sizeof(h), cudaMemcpyDeviceToHost, s));
+  CU(ctx, cudaMemsetAsync(dev_status(ctx), 0, sizeof(DevStatus), s));
+  CU(ctx, cudaStreamSynchronize(s));
+  if (h.timeout) return AGZO_ERR_TIMEOUT;
+  if (h.rank_deficient) return AGZO_WARN_RANK_DEFICIENT;
+  return AGZO_OK;
+}
+
+agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                                  int K, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (K < 0 || K > 16) return AGZO_ERR_INVALID_ARG;
+  st = validate(h_layers, n, NEED_EXTRACT);
+  if (st != AGZO_OK) return st;
+  if (n == 0) return AGZO_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->extract_path == 2)
+    for (int i = 0; i < n; ++i)
+      if (!tc_eligible(h_layers[i])) return AGZO_ERR_UNSUPPORTED;
+  st = prepare(ctx, h_layers, n, s);
+  if (st != AGZO_OK) return st;
+
+  const Plan& P = ctx->plan;
+  int l0 = 0;
+  for (size_t wv = 0; wv < P.wave_end.size(); ++wv) {
+    const int l1 = P.wave_end[wv];
+    ExtractWave w{};
+    w.d_layers = dev_layers(ctx);
+    w.l0 = l0; w.l1 = l1;
+    bool all_tc = ctx->extract_path != 1;
+    for (int i = l0; i < l1; ++i) {
+      const DevLayer& D = P.dev[i];
+      if (D.m > w.max_m) w.max_m = D.m;
+      if (D.d_in > w.max_din) w.max_din = D.d_in;
+      if (D.r > w.max_r) w.max_r = D.r;
+      if (D.slabs > w.max_slabs) w.max_slabs = D.slabs;
+      if (D.gchunks > w.max_gchunks) w.max_gchunks = D.gchunks;
+      if (!D.Qb) all_tc = false;
+    }
+    l0 = l1;
+    if (w.max_m == 0) continue;
+    DevStatus* dst = dev_status(ctx);
+    if (all_tc) {
+      // tensor-core products; the panel factorisation is shared
+      CU(ctx, tc_fill_omega(ctx->tc, w, P.dev.data(), seed, s));
+      CU(ctx, tc_xt_t(ctx->tc, w, P.dev.data(), dst, s));
+      for (int k = 0; k < K; ++k) {
+        CU(ctx, launch_panel_qr(w, dst, s));
+        CU(ctx, tc_x_q(ctx->tc, w, P.dev.data(), dst, s));
+        CU(ctx, tc_xt_t(ctx->tc, w, P.dev.data(), dst, s));
+      }
+      CU(ctx, launch_panel_qr(w, dst, s));
+    } else {
+      CU(ctx, launch_fill_omega(w, seed, s));
+      CU(ctx, launch_xt_t(w, s));
+      for (int k = 0; k < K; ++k) {
+        CU(ctx, launch_panel_qr(w, dst, s));
+        CU(ctx, launch_x_q(w, s));
+        CU(ctx, launch_xt_t(w, s));
+      }
+      CU(ctx, launch_panel_qr(w, dst, s));
+    }
+  }
+  return AGZO_OK;
+}
+
+agzo_status agzo_perturb(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                         float scale, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  return rmw_pass(ctx, h_layers, n, seed, scale, nullptr, false, static_cast<cudaStream_t>(stream));
+}
+
+agzo_status agzo_restore(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                         float scale, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  // a master/compute pair is restored by rewriting W16 = bf16(W): coefficient 0 on the pair path
+  bool any_pair = false, any_plain = false;
+  for (int i = 0; h_layers && i < n; ++i) (h_layers[i].W16 ? any_pair : any_plain) = true;
+  if (any_pair && any_plain) return AGZO_ERR_UNSUPPORTED;
+  const float c = any_pair ? 0.0f : -scale;
+  return rmw_pass(ctx, h_layers, n, seed, c, nullptr, false, static_cast<cudaStream_t>(stream));
+}
+
+agzo_status agzo_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed, float lr,
+                        const float* d_ghat, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!d_ghat) return AGZO_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = validate(h_layers, n, NEED_RMW);
+  if (st != AGZO_OK) return st;
+  if (n == 0) return AGZO_OK;
+  CU(ctx, launch_coef(d_ghat, 0.f, lr, 2, dev_coef(ctx), s));
+  return rmw_pass(ctx, h_layers, n, seed, 0.f, dev_coef(ctx), true, s);
+}
+
+agzo_status agzo_ghat(agzo_ctx* ctx, const float* d_f_plus, const float* d_f_other, float eps,
+                      int mode, float* d_ghat, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!d_f_plus || !d_f_other || !d_ghat || !(eps > 0.f) || (mode != 0 && mode != 1))
+    return AGZO_ERR_INVALID_ARG;
+  CU(ctx, launch_ghat(d_f_plus, d_f_other, eps, mode, d_ghat, static_cast<cudaStream_t>(stream)));
+  return AGZO_OK;
+}
+
+agzo_status agzo_restore_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                                float eps, float lr, int mode, const float* d_ghat, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!d_ghat || (mode != 0 && mode != 1)) return AGZO_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = validate(h_layers, n, NEED_RMW);
+  if (st != AGZO_OK) return st;
+  if (n == 0) return AGZO_OK;
+  bool any_pair = false, any_plain = false;
+  for (int i = 0; i < n; ++i) (h_layers[i].W16 ? any_pair : any_plain) = true;
+  if (any_pair && any_plain) return AGZO_ERR_UNSUPPORTED;
+  // a pair's master was never perturbed: only the update term applies to it
+  CU(ctx, launch_coef(d_ghat, eps, lr, any_pair ? 2 : mode, dev_coef(ctx), s));
+  return rmw_pass(ctx, h_layers, n, seed, 0.f, dev_coef(ctx), true, s);
+}
+
+agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n, const agzo_params* p,
+                      agzo_loss_fn loss, void* user, float* d_out3, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!p || !loss || !d_out3 || !(p->eps > 0.f) || (p->mode != 0 && p->mode != 1) || p->K < 0 ||
+      p->K > 16)
+    return AGZO_ERR_INVALID_ARG;
+  st = validate(h_layers, n, NEED_RMW | NEED_EXTRACT);
+  if (st != AGZO_OK) return st;
+  bool any_pair = false, any_plain = false;
+  for (int i = 0; i < n; ++i) (h_layers[i].W16 ? any_pair : any_plain) = true;
+  if (any_pair && any_plain) return AGZO_ERR_UNSUPPORTED;
+  float* d_fplus = d_out3;
+  float* d_fother = d_out3 + 1;
+  float* d_g = d_out3 + 2;
+
+  // step 1: unperturbed forward (fills X), then Algorithm 1 per layer
+  if (loss(user, stream, 0, d_fother) != 0) return AGZO_ERR_CALLBACK;
+  st = agzo_extract_subspace(ctx, h_layers, n, p->seed, p->K, stream);
+  if (st != AGZO_OK) return st;
+  // step 2: W + eps*Delta
+  st = agzo_perturb(ctx, h_layers, n, p->seed, p->eps, stream);
+  if (st != AGZO_OK) return st;
+  if (loss(user, stream, 1, d_fplus) != 0) {
+    agzo_restore(ctx, h_layers, n, p->seed, p->eps, stream);
+    return AGZO_ERR_CALLBACK;
+  }
+  if (p->mode == 0) {
+    // a pair is always rebuilt from the untouched master, so its flip is -eps, not -2 eps
+    st = agzo_perturb(ctx, h_layers, n, p->seed, any_pair ? -p->eps : -2.0f * p->eps, stream);
+    if (st != AGZO_OK) return st;
+    if (loss(user, stream, 2, d_fother) != 0) {
+      agzo_restore(ctx, h_layers, n, p->seed, -p->eps, stream);
+      return AGZO_ERR_CALLBACK;
+    }
+  }
+  st = agzo_ghat(ctx, d_fplus, d_fother, p->eps, p->mode, d_g, stream);
+  if (st != AGZO_OK) return st;
+  // step 3: restore and update in one pass
+  return agzo_restore_update(ctx, h_layers, n, p->seed, p->eps, p->lr, p->mode, d_g, stream);
+}
+
+agzo_status agzo_perturb_dense(agzo_ctx* ctx, void* w, int64_t n_elems, int dtype, uint64_t seed,
+                               uint32_t layer_id, float scale, const float* d_scale, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (n_elems < 0 || (n_elems > 0 && !w)) return AGZO_ERR_INVALID_ARG;
+  if (dtype != AGZO_BF16 && dtype != AGZO_F32) return AGZO_ERR_UNSUPPORTED;
+  CU(ctx, launch_dense(w, n_elems, dtype, seed, layer_id, scale, d_scale,
+                       static_cast<cudaStream_t>(stream)));
+  return AGZO_OK;
+}
+
+agzo_status agzo_debug_philox(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, uint32_t tag,
+                              uint64_t first, uint64_t n, uint32_t* d_words, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (n > 0 && !d_words) return AGZO_ERR_INVALID_ARG;
+  CU(ctx, launch_debug_philox(seed, layer_id, tag, first, n, d_words, static_cast<cudaStream_t>(stream)));
+  return AGZO_OK;
+}
+
+agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, uint32_t tag,
+                                uint64_t first, uint64_t n, float* d_vals, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (n > 0 && !d_vals) return AGZO_ERR_INVALID_ARG;
+  CU(ctx, launch_debug_gauss(seed, layer_id, tag, first, n, d_vals, static_cast<cudaStream_t>(stream)));
+  return AGZO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,292 @@
+// Algorithm 1 (SubspaceExtract) on CUDA cores in fp32, plus the panel orthonormalisation
+// that both extraction paths share.  This path takes any dtype, pitch and size; the
+// tensor-core path (agzo_extract_tc.cu) replaces the two products with X when the layer's
+// shape allows it.
+//
+// Products:  Ypart[s] = X_s^T T_s  per token slab s (summed in slab order later, so the result
+//            does not depend on scheduling), and T = X Q.
+// qr(Y):     Gram matrix S = Y^T Y accumulated in double, Cholesky S = R^T R with R_kk > 0,
+//            Q = Y R^-1.  With the Gram matrix and the factor in double this is as accurate
+//            in fp32 as a Householder QR for cond(Y) well below 1e7, and it is the unique
+//            positive-diagonal factorisation that the method's definition fixes.
+#include "agzo_common.cuh"
+
+namespace agzo {
+
+// ------------------------------------------------------------------ Omega -> T
+__global__ void fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const long long n = (long long)L.m * L.r;
+  const long long nb = (n + 3) >> 2;
+  for (long long b = blockIdx.x * (long long)blockDim.x + threadIdx.x; b < nb;
+       b += (long long)gridDim.x * blockDim.x) {
+    const float4 g = gaussian_block((uint64_t)b, L.layer_id, kTagOmega, seed);
+    const float gv[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+    for (int lane = 0; lane < 4; ++lane) {
+      const long long e = 4 * b + lane;
+      if (e < n) L.T[e] = gv[lane];
+    }
+  }
+}
+
+cudaError_t launch_fill_omega(const ExtractWave& w, uint64_t seed, cudaStream_t s) {
+  const long long nb = ((long long)w.max_m * w.max_r + 3) >> 2;
+  int gx = (int)((nb + 255) / 256);
+  if (gx > 512) gx = 512;
+  if (gx < 1) gx = 1;
+  fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed);
+  return cudaGetLastError();
+}
+
+__device__ __forceinline__ float load_x(const DevLayer& L, long long t, int d) {
+  return L.x_dtype == AGZO_BF16
+             ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(L.X)[t * L.ldx + d])
+             : reinterpret_cast<const float*>(L.X)[t * L.ldx + d];
+}
+
+// ------------------------------------------------------------------ Ypart[s][k][d] = sum_{t in slab s} X[t][d] T[t][k]
+// block: 256 threads = 256 columns d; grid (d chunks, slabs, layers).  Rank handled in chunks of 16.
+constexpr int kXtTokens = 32;
+__global__ void __launch_bounds__(256) xt_t_kernel(const DevLayer* __restrict__ layers, int l0) {
+  const DevLayer& L = layers[l0 + blockIdx.z];
+  const int slab = blockIdx.y;
+  if (slab >= L.slabs) return;
+  const int d0 = blockIdx.x * 256;
+  if (d0 >= L.d_in) return;
+  const int d = d0 + threadIdx.x;
+  const bool d_ok = d < L.d_in;
+  const int t_begin = slab * L.slab_rows;
+  const int t_end = min(L.m, t_begin + L.slab_rows);
+  __shared__ float sT[kXtTokens][16];
+  const int r = L.r;
+  for (int k0 = 0; k0 < r; k0 += 16) {
+    const int kc = min(16, r - k0);
+    float acc[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+    for (int tb = t_begin; tb < t_end; tb += kXtTokens) {
+      __syncthreads();
+      for (int i = threadIdx.x; i < kXtTokens * 16; i += 256) {
+        const int tt = i >> 4, k = i & 15;
+        sT[tt][k] = (tb + tt < t_end && k < kc) ? L.T[(long long)(tb + tt) * r + k0 + k] : 0.f;
+      }
+      __syncthreads();
+      if (d_ok) {
+        const int nt = min(kXtTokens, t_end - tb);
+        for (int tt = 0; tt < nt; ++tt) {
+          const float x = load_x(L, tb + tt, d);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) acc[k] = fmaf(x, sT[tt][k], acc[k]);
+        }
+      }
+    }
+    if (d_ok) {
+      float* out = L.Ypart + ((long long)slab * r + k0) * L.d_in + d;
+      for (int k = 0; k < kc; ++k) out[(long long)k * L.d_in] = acc[k];
+    }
+  }
+}
+
+cudaError_t launch_xt_t(const ExtractWave& w, cudaStream_t s) {
+  dim3 grid((w.max_din + 255) / 256, w.max_slabs, w.l1 - w.l0);
+  xt_t_kernel<<<grid, 256, 0, s>>>(w.d_layers, w.l0);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ T[t][k] = sum_d X[t][d] Q[k][d]   (Q = rows of V)
+// one warp per token; Q streamed through shared memory in column chunks.
+constexpr int kXqCols = 256;
+constexpr int kXqWarps = 8;
+__global__ void __launch_bounds__(256) x_q_kernel(const DevLayer* __restrict__ layers, int l0) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tokens_per_block = kXqWarps * 4;
+  const int t0 = blockIdx.x * tokens_per_block;
+  if (t0 >= L.m) return;
+  __shared__ float sQ[16][kXqCols + 1];
+  const int r = L.r;
+  for (int k0 = 0; k0 < r; k0 += 16) {
+    const int kc = min(16, r - k0);
+    float acc[4][16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int k = 0; k < 16; ++k) acc[i][k] = 0.f;
+    for (int c0 = 0; c0 < L.d_in; c0 += kXqCols) {
+      __syncthreads();
+      for (int i = threadIdx.x; i < 16 * kXqCols; i += 256) {
+        const int k = i / kXqCols, c = i - k * kXqCols;
+        sQ[k][c] = (k < kc && c0 + c < L.d_in) ? L.V[(long long)(k0 + k) * L.ldv + c0 + c] : 0.f;
+      }
+      __syncthreads();
+      const int nc = min(kXqCols, L.d_in - c0);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int t = t0 + warp * 4 + i;
+        if (t < L.m) {
+          for (int c = lane; c < nc; c += 32) {
+            const float x = load_x(L, t, c0 + c);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) acc[i][k] = fmaf(x, sQ[k][c], acc[i][k]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int t = t0 + warp * 4 + i;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        float v = acc[i][k];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0 && t < L.m && k < kc) L.T[(long long)t * r + k0 + k] = v;
+      }
+    }
+  }
+}
+
+cudaError_t launch_x_q(const ExtractWave& w, cudaStream_t s) {
+  dim3 grid((w.max_m + kXqWarps * 4 - 1) / (kXqWarps * 4), w.l1 - w.l0);
+  x_q_kernel<<<grid, 256, 0, s>>>(w.d_layers, w.l0);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ qr(Y), stage 1
+// Y[k][d] = sum_s Ypart[s][k][d] (fixed order) and the partial Gram matrix of this block's
+// column chunk in double.  block = 128 columns.
+constexpr int kGramCols = 128;
+__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const int chunk = blockIdx.x;
+  if (chunk >= L.gchunks) return;
+  extern __shared__ __align__(16) float sY[];   // [r][kGramCols]
+  const int r = L.r;
+  const int d0 = chunk * kGramCols;
+  for (int i = threadIdx.x; i < r * kGramCols; i += 256) {
+    const int k = i / kGramCols, c = i - k * kGramCols;
+    const int d = d0 + c;
+    float y = 0.f;
+    if (d < L.d_in) {
+      for (int s = 0; s < L.slabs; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
+      L.Y[(long long)k * L.d_in + d] = y;
+    }
+    sY[i] = y;
+  }
+  __syncthreads();
+  double* out = L.Gpart + (long long)chunk * r * r;
+  for (int p = threadIdx.x; p < r * r; p += 256) {
+    const int i = p / r, j = p - i * r;
+    if (j < i) continue;
+    double acc = 0.0;
+    const float* yi = sY + i * kGramCols;
+    const float* yj = sY + j * kGramCols;
+    for (int c = 0; c < kGramCols; ++c) acc = fma((double)yi[c], (double)yj[c], acc);
+    out[i * r + j] = acc;
+  }
+}
+
+// ------------------------------------------------------------------ qr(Y), stage 2: one block per layer
+// S = sum of partial Gram matrices; Cholesky S = R^T R (upper R, positive diagonal); a pivot
+// with R_kk <= kRankTol * R_11 marks a deficient column, which becomes zero.  M (upper
+// triangular) is built so that Q = Y M: column k of M solves R-columns by forward substitution.
+__global__ void __launch_bounds__(64) chol_kernel(const DevLayer* __restrict__ layers, int l0,
+                                                  DevStatus* status) {
+  const DevLayer& L = layers[l0 + blockIdx.x];
+  const int r = L.r;
+  __shared__ double S[AGZO_MAX_RANK][AGZO_MAX_RANK + 1];
+  __shared__ int bad[AGZO_MAX_RANK];
+  __shared__ double piv;
+  double* Mm = L.M;                     // [r][r], written and re-read by this block only
+  const int tid = threadIdx.x;
+  for (int p = tid; p < r * r; p += 64) {
+    const int i = p / r, j = p - i * r;
+    double acc = 0.0;
+    if (j >= i)
+      for (int c = 0; c < L.gchunks; ++c) acc += L.Gpart[(long long)c * r * r + p];
+    S[i][j] = acc;
+    Mm[p] = 0.0;
+  }
+  __syncthreads();
+  // right-looking Cholesky on the upper triangle; S is overwritten by R
+  for (int k = 0; k < r; ++k) {
+    if (tid == 0) {
+      const double d = S[k][k];
+      const double r11 = k == 0 ? 0.0 : S[0][0];
+      int b = 0;
+      if (!(d > 0.0)) b = 1;
+      else if (k > 0 && sqrt(d) <= (double)kRankTol * r11) b = 1;
+      bad[k] = b;
+      piv = b ? 0.0 : sqrt(d);
+      S[k][k] = piv;
+      if (b) atomicExch(&status->rank_deficient, 1);
+    }
+    __syncthreads();
+    const double pk = piv;
+    for (int j = k + 1 + tid; j < r; j += 64) S[k][j] = pk > 0.0 ? S[k][j] / pk : 0.0;
+    __syncthreads();
+    const int nn = r - k - 1;
+    for (int p = tid; p < nn * nn; p += 64) {
+      const int i = k + 1 + p / nn, j = k + 1 + p % nn;
+      if (j >= i) S[i][j] -= S[k][i] * S[k][j];
+    }
+    __syncthreads();
+  }
+  // M column by column: M[row][k] = (delta_{row,k} - sum_{row<=i<k} M[row][i] R[i][k]) / R[k][k];
+  // a deficient column stays zero
+  for (int k = 0; k < r; ++k) {
+    if (!bad[k]) {
+      for (int row = tid; row <= k; row += 64) {
+        double acc = row == k ? 1.0 : 0.0;
+        for (int i = row; i < k; ++i) acc -= Mm[row * r + i] * S[i][k];
+        Mm[row * r + k] = acc / S[k][k];
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------ qr(Y), stage 3: Q = Y M
+// thread per column d; writes Q (fp32) into V and, for the tensor-core path, the bf16
+// hi/lo panels.
+__global__ void __launch_bounds__(128) apply_kernel(const DevLayer* __restrict__ layers, int l0) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const int d = blockIdx.x * 128 + threadIdx.x;
+  extern __shared__ __align__(16) double sM[];   // [r][r]
+  const int r = L.r;
+  for (int p = threadIdx.x; p < r * r; p += 128) sM[p] = L.M[p];
+  __syncthreads();
+  if (d >= L.d_in || blockIdx.x * 128 >= L.d_in) return;
+  float y[AGZO_MAX_RANK];
+#pragma unroll 4
+  for (int j = 0; j < r; ++j) y[j] = L.Y[(long long)j * L.d_in + d];
+  for (int k = 0; k < r; ++k) {
+    double acc = 0.0;
+    for (int j = 0; j <= k; ++j) acc = fma((double)y[j], sM[j * r + k], acc);
+    const float q = (float)acc;
+    L.V[(long long)k * L.ldv + d] = q;
+    if (L.Qb) {
+      const __nv_bfloat16 hi = __float2bfloat16_rn(q);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(q - __bfloat162float(hi));
+      L.Qb[(long long)k * L.d_in + d] = hi;
+      L.Qb[(long long)(L.NP + k) * L.d_in + d] = lo;
+    }
+  }
+}
+
+cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s) {
+  const int nl = w.l1 - w.l0;
+  reduce_gram_kernel<<<dim3(w.max_gchunks, nl), 256, (size_t)w.max_r * kGramCols * sizeof(float), s>>>(
+      w.d_layers, w.l0);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  chol_kernel<<<nl, 64, 0, s>>>(w.d_layers, w.l0, d_status);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  apply_kernel<<<dim3((w.max_din + 127) / 128, nl), 128, (size_t)w.max_r * w.max_r * sizeof(double), s>>>(
+      w.d_layers, w.l0);
+  return cudaGetLastError();
+}
+
+}  // namespace agzo

@@ -1,0 +1,80 @@
+"""Shared pieces of the GPU parity tests: upload seeded host data, run the library through
+its C ABI, bring results back, compare with the oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import agzo_oracle as O
+from paper_2601_17261_b200 import binding as B
+
+DEV = "cuda:0"
+
+
+def to_dev(x: np.ndarray, bf16: bool, pitch: int | None = None, fill: float = 7.0):
+    """Uploads a 2-D float32 array; with `pitch` the rows sit in a wider buffer whose padding
+    holds a sentinel (returns (view, whole buffer))."""
+    dt = torch.bfloat16 if bf16 else torch.float32
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32))
+    if pitch is None:
+        d = t.to(DEV).to(dt).contiguous()
+        return d, d
+    buf = torch.full((x.shape[0] + 2, pitch), fill, dtype=dt, device=DEV)
+    view = buf[1:1 + x.shape[0], : x.shape[1]]
+    view.copy_(t.to(DEV).to(dt))
+    return view, buf
+
+
+def to_host(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy()
+
+
+def bf16_ulp_distance(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """Distance in bf16 steps between two arrays of bf16-representable float32 values."""
+    def key(x):
+        u = O.f32_to_bf16_bits(x).astype(np.int32)
+        return np.where(u & 0x8000, 0x8000 - u, u)   # monotone integer order
+    return np.abs(key(a) - key(b))
+
+
+def f32_ulp_distance(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    def key(x):
+        u = np.ascontiguousarray(x, dtype=np.float32).view(np.int32).astype(np.int64)
+        return np.where(u < 0, -(u & 0x7FFFFFFF), u)
+    return np.abs(key(a) - key(b))
+
+
+def projector_distance(Va: np.ndarray, Vb: np.ndarray) -> float:
+    """|| Va^T Va - Vb^T Vb ||_F for V stored as r rows of length d_in, without forming the
+    d_in x d_in projectors: ||Pa - Pb||^2 = ||Va Va^T||^2 + ||Vb Vb^T||^2 - 2 ||Va Vb^T||^2."""
+    Va = Va.astype(np.float64)
+    Vb = Vb.astype(np.float64)
+    a = np.linalg.norm(Va @ Va.T) ** 2
+    b = np.linalg.norm(Vb @ Vb.T) ** 2
+    c = np.linalg.norm(Va @ Vb.T) ** 2
+    return float(np.sqrt(max(a + b - 2 * c, 0.0)))
+
+
+def assert_weights_match(got: np.ndarray, want: np.ndarray, storage: str, frac: float = 1e-3):
+    """<= 1 bf16 ulp everywhere (<= 4 fp32 ulp for fp32 storage), mismatches rare."""
+    if storage == "bf16":
+        d = bf16_ulp_distance(got, want)
+        assert d.max() <= 1, f"max bf16 ulp distance {d.max()}"
+    else:
+        d = f32_ulp_distance(got, want)
+        assert d.max() <= 4, f"max fp32 ulp distance {d.max()}"
+    assert (d > 0).mean() <= frac, f"mismatching fraction {(d > 0).mean()}"
+
+
+class Ctx:
+    """Context sized for a layer list, destroyed on exit."""
+
+    def __init__(self, layers, extra=0):
+        self.ctx = B.agzo_create(layers, 0, extra)
+
+    def __enter__(self):
+        return self.ctx
+
+    def __exit__(self, *a):
+        torch.cuda.synchronize()
+        B.agzo_destroy(self.ctx)

@@ -1,0 +1,292 @@
+"""GPU-vs-oracle parity through the C ABI, on seeded inputs.
+
+Tolerances (stated as numbers):
+  Philox words and the element -> (block, lane) map ........ bit-exact
+  normals ................................................... |d| <= 2e-6 * max(1, |g|)
+  V (projector) ............................................. ||VtV_gpu - VtV_cpu||_F <= 1e-3
+  V orthonormality .......................................... max |V V^T - I| <= 1e-5
+  bf16 weights after a pass (same V on both sides) .......... <= 1 bf16 ulp, <= 1e-3 of them differ
+  fp32 weights .............................................. <= 4 fp32 ulp
+  ghat ...................................................... 1e-3 relative
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import agzo_oracle as O
+from paper_2601_17261_b200 import binding as B
+from paper_2601_17261_b200 import workloads as WL
+
+from gpu_helpers import (DEV, Ctx, assert_weights_match, bf16_ulp_distance, projector_distance,
+                         to_dev, to_host)
+
+pytestmark = pytest.mark.gpu
+
+
+# ----------------------------------------------------------------------------- generator
+def test_philox_words_bit_exact():
+    V = torch.zeros(1, 8, device=DEV)
+    with Ctx([B.make_layer(V=V, r=1, layer_id=0, d_in=8)]) as ctx:
+        for seed, layer, tag, first, n in [(0, 0, 0, 0, 4099), (0xDEADBEEFCAFEF00D, 251, 1, 0, 1000),
+                                           (7, 3, 2, (1 << 34) + 5, 257), (1, 0xFFFFFFFF, 0, 3, 64)]:
+            got = B.agzo_debug_philox(ctx, seed, layer, tag, first, n).cpu().numpy().view(np.uint32)
+            want = O.philox_words(seed, layer, tag, n, first=first)
+            assert np.array_equal(got, want)
+        assert B.agzo_debug_philox(ctx, 1, 1, 1, 0, 0).numel() == 0
+
+
+def test_gaussians_match_the_oracle():
+    V = torch.zeros(1, 8, device=DEV)
+    with Ctx([B.make_layer(V=V, r=1, layer_id=0, d_in=8)]) as ctx:
+        n = 1 << 20
+        for seed, layer, tag in [(0, 0, 0), (12345678901234, 17, 1), (3, 9, 2)]:
+            got = B.agzo_debug_gaussian(ctx, seed, layer, tag, 0, n).cpu().numpy()
+            want = O.gaussian_stream(seed, layer, tag, n)
+            err = np.abs(got.astype(np.float64) - want) / np.maximum(1.0, np.abs(want))
+            assert err.max() <= 2e-6
+
+
+# ----------------------------------------------------------------------------- in-place passes
+RMW_CASES = [
+    # d_out, d_in, r, storage, pitch_extra, label
+    (300, 1024, 8, "bf16", 0, "two column tiles, ragged rows"),
+    (257, 520, 4, "bf16", 8, "ragged tile edge, padded pitch"),
+    (64, 256, 1, "bf16", 0, "r=1"),
+    (130, 512, 2, "bf16", 0, "r=2"),
+    (96, 768, 3, "bf16", 0, "r=3 (padded rank chunk)"),
+    (520, 1536, 16, "bf16", 0, "r=16"),
+    (300, 640, 24, "bf16", 0, "r=24 shared-memory kernel"),
+    (260, 512, 64, "bf16", 0, "r=64"),
+    (256, 256, 4, "f32", 0, "fp32 storage"),
+    (100, 136, 8, "f32", 4, "fp32 padded pitch"),
+    (37, 50, 5, "bf16", 1, "unaligned: scalar kernel"),
+    (19, 27, 3, "f32", 0, "unaligned fp32"),
+]
+
+
+@pytest.mark.parametrize("d_out,d_in,r,storage,extra,label", RMW_CASES)
+def test_perturb_restore_update_match_oracle(d_out, d_in, r, storage, extra, label):
+    seed, layer_id = 11, 5
+    bf = storage == "bf16"
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=d_out + d_in, bf16=bf)
+    Vh = O.extract_subspace(WL.plain_activations(max(2 * r, 32), d_in, seed=r), r, 1, 3, layer_id)
+    Wd, Wbuf = to_dev(W0, bf, pitch=d_in + extra if extra else None)
+    Vd, Vbuf = to_dev(Vh, False, pitch=d_in + (4 if extra else 0) if extra else None)
+    layers = [B.make_layer(W=Wd, V=Vd, r=r, layer_id=layer_id)]
+    ghat = torch.tensor([0.73], device=DEV)
+    with Ctx(layers) as ctx:
+        eps = 1e-3
+        B.agzo_perturb(ctx, layers, seed, eps)
+        want = O.apply_direction(W0, Vh, seed, layer_id, np.float32(eps), storage)
+        assert_weights_match(to_host(Wd), want, storage)
+        B.agzo_perturb(ctx, layers, seed, -2 * eps)
+        want = O.apply_direction(want, Vh, seed, layer_id, np.float32(-2 * eps), storage)
+        assert_weights_match(to_host(Wd), want, storage, frac=2e-3)
+        # feed the oracle the GPU's weights from here on so that mismatches do not compound
+        cur = to_host(Wd)
+        B.agzo_restore(ctx, layers, seed, -eps)
+        want = O.apply_direction(cur, Vh, seed, layer_id, np.float32(eps), storage)
+        assert_weights_match(to_host(Wd), want, storage)
+        cur = to_host(Wd)
+        B.agzo_update(ctx, layers, seed, 5e-2, ghat)
+        want = O.apply_direction(cur, Vh, seed, layer_id, np.float32(-5e-2 * np.float32(0.73)), storage)
+        assert_weights_match(to_host(Wd), want, storage)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    if extra:  # the padding around W and V is untouched
+        w = Wbuf.float()
+        assert bool((w[0] == 7).all() and (w[-1] == 7).all() and (w[:, d_in:] == 7).all())
+        assert bool((Vbuf[0] == 7).all() and (Vbuf[:, d_in:] == 7).all())
+
+
+def test_restore_update_fused_modes():
+    d_out, d_in, r, seed = 200, 512, 8, 21
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=1, bf16=True)
+    Vh = O.extract_subspace(WL.plain_activations(64, d_in, seed=2), r, 1, 3, 0)
+    Vd, _ = to_dev(Vh, False)
+    g = np.float32(-1.37)
+    ghat = torch.tensor([float(g)], device=DEV)
+    for mode in (0, 1):
+        Wd, _ = to_dev(W0, True)
+        layers = [B.make_layer(W=Wd, V=Vd, r=r, layer_id=0)]
+        with Ctx(layers) as ctx:
+            B.agzo_restore_update(ctx, layers, seed, 1e-3, 2e-3, mode, ghat)
+            c = O.update_coefficient(1e-3, 2e-3, g, mode)
+            want = O.apply_direction(W0, Vh, seed, 0, c, "bf16")
+            assert_weights_match(to_host(Wd), want, "bf16")
+
+
+def test_many_layers_one_launch_mixed_shapes_and_ranks():
+    rng = np.random.default_rng(0)
+    shapes = [(128, 256, 2), (300, 512, 8), (64, 1024, 8), (257, 264, 5), (33, 40, 3), (512, 512, 1)]
+    host, layers, devW = [], [], []
+    for i, (do, di, r) in enumerate(shapes):
+        W0 = WL.gaussian_weights(do, di, 0.02, seed=i, bf16=True)
+        Vh = O.extract_subspace(WL.plain_activations(32, di, seed=i), r, 1, 9, 100 + i)
+        Wd, _ = to_dev(W0, True)
+        Vd, _ = to_dev(Vh, False)
+        host.append((W0, Vh, r))
+        devW.append((Wd, Vd))
+        layers.append(B.make_layer(W=Wd, V=Vd, r=r, layer_id=100 + i))
+    with Ctx(layers) as ctx:
+        B.agzo_perturb(ctx, layers, 77, 2e-3)
+        for i, (W0, Vh, r) in enumerate(host):
+            want = O.apply_direction(W0, Vh, 77, 100 + i, np.float32(2e-3), "bf16")
+            assert_weights_match(to_host(devW[i][0]), want, "bf16", frac=2e-3)
+
+
+def test_perturb_is_deterministic_and_regenerates_the_same_direction():
+    d_out, d_in, r = 512, 1024, 8
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=3, bf16=False)
+    Vh = O.extract_subspace(WL.plain_activations(64, d_in, seed=2), r, 1, 3, 0)
+    Vd, _ = to_dev(Vh, False)
+    outs = []
+    for _ in range(2):
+        Wd, _ = to_dev(W0, False)
+        layers = [B.make_layer(W=Wd, V=Vd, r=r, layer_id=1)]
+        with Ctx(layers) as ctx:
+            B.agzo_perturb(ctx, layers, 5, 1e-2)
+            outs.append(to_host(Wd))
+            B.agzo_restore(ctx, layers, 5, 1e-2)
+            back = to_host(Wd)
+    assert np.array_equal(outs[0], outs[1])
+    assert np.abs(back - W0).max() < 1e-8     # fp32: W + cZ - cZ returns to W within rounding
+
+
+def test_dense_direction():
+    w0 = WL.gaussian_weights(1, 100003, 0.5, seed=9, bf16=True).reshape(-1)
+    wd = torch.from_numpy(w0).to(DEV).to(torch.bfloat16)
+    V = torch.zeros(1, 8, device=DEV)
+    scale = torch.tensor([-2.0], device=DEV)
+    with Ctx([B.make_layer(V=V, r=1, layer_id=0, d_in=8)]) as ctx:
+        B.agzo_perturb_dense(ctx, wd, 4, 33, 1e-2)
+        want = O.apply_dense(w0, 4, 33, np.float32(1e-2), "bf16")
+        d = bf16_ulp_distance(to_host(wd), want)
+        assert d.max() <= 1 and (d > 0).mean() < 1e-3
+        w1 = to_host(wd)
+        B.agzo_perturb_dense(ctx, wd, 4, 33, 1e-2, d_scale=scale)
+        want = O.apply_dense(w1, 4, 33, np.float32(-2e-2), "bf16")
+        d = bf16_ulp_distance(to_host(wd), want)
+        assert d.max() <= 1 and (d > 0).mean() < 1e-3
+
+
+def test_ghat_scalar():
+    V = torch.zeros(1, 8, device=DEV)
+    fp = torch.tensor([0.731234], device=DEV)
+    fo = torch.tensor([0.729876], device=DEV)
+    g = torch.zeros(1, device=DEV)
+    with Ctx([B.make_layer(V=V, r=1, layer_id=0, d_in=8)]) as ctx:
+        B.agzo_ghat(ctx, fp, fo, 1e-3, 0, g)
+        want = O.ghat_two_point(np.float32(0.731234), np.float32(0.729876), 1e-3)
+        assert abs(g.item() - float(want)) <= 1e-6 * abs(float(want))
+        B.agzo_ghat(ctx, fp, fo, 1e-3, 1, g)
+        want = O.ghat_one_sided(np.float32(0.731234), np.float32(0.729876), 1e-3)
+        assert abs(g.item() - float(want)) <= 1e-6 * abs(float(want))
+
+
+# ----------------------------------------------------------------------------- Algorithm 1
+EXTRACT_CASES = [
+    # m, d_in, r, K, planted, x_bf16, path
+    (512, 256, 4, 3, 0, False, 1),       # the single-layer fp32 problem's shape
+    (700, 520, 8, 3, 16, True, 1),       # ragged everything
+    (1000, 384, 1, 3, 8, True, 1),
+    (333, 200, 16, 2, 32, True, 1),
+    (2048, 1024, 8, 3, 32, True, 1),
+    (640, 256, 24, 1, 32, True, 1),
+    (300, 128, 64, 1, 0, False, 1),
+    (400, 96, 5, 0, 0, False, 1),        # K = 0: just qr(H Omega)
+]
+
+
+def _run_extract(X, r, K, seed, layer_id, path, x_bf16, pitch=None):
+    Xd, _ = to_dev(X, x_bf16, pitch=pitch)
+    Vd = torch.full((r + 2, X.shape[1] + 4), 7.0, device=DEV)
+    Vv = Vd[1:1 + r, : X.shape[1]]
+    layers = [B.make_layer(X=Xd, V=Vv, r=r, layer_id=layer_id)]
+    with Ctx(layers) as ctx:
+        B.agzo_set_option(ctx, "extract_path", path)
+        B.agzo_extract_subspace(ctx, layers, seed, K)
+        st = B.agzo_poll(ctx)
+    assert bool((Vd[0] == 7).all() and (Vd[-1] == 7).all() and (Vd[:, X.shape[1]:] == 7).all())
+    return to_host(Vv), st
+
+
+@pytest.mark.parametrize("m,d_in,r,K,planted,x_bf16,path", EXTRACT_CASES)
+def test_extract_matches_oracle(m, d_in, r, K, planted, x_bf16, path):
+    X = (WL.planted_activations(m, d_in, planted, seed=m, bf16=x_bf16) if planted
+         else WL.plain_activations(m, d_in, seed=m, bf16=x_bf16))
+    Vg, st = _run_extract(X, r, K, seed=13, layer_id=4, path=path, x_bf16=x_bf16,
+                          pitch=d_in + 8 if d_in % 16 else None)
+    assert st == B.AGZO_OK
+    Vo = O.extract_subspace(X, r, K, 13, 4)
+    assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
+    assert projector_distance(Vg, Vo) <= 1e-3
+    assert np.abs(Vg - Vo).max() <= 1e-3          # the basis itself, not only its span
+
+
+def test_extract_many_layers_in_waves():
+    specs = [(600, 256, 4), (512, 512, 8), (900, 128, 2), (512, 256, 8), (384, 320, 6)]
+    Xs = [WL.planted_activations(m, d, 16, seed=i, bf16=True) for i, (m, d, r) in enumerate(specs)]
+    devs, layers = [], []
+    for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
+        Xd, _ = to_dev(X, True)
+        Vd = torch.zeros(r, d, device=DEV)
+        devs.append((Xd, Vd))
+        layers.append(B.make_layer(X=Xd, V=Vd, r=r, layer_id=i))
+    for wave_bytes in (1 << 30, 400 * 1024, 1):      # one wave, several, one layer per wave
+        with Ctx(layers) as ctx:
+            B.agzo_set_option(ctx, "extract_path", 1)
+            B.agzo_set_option(ctx, "wave_bytes", wave_bytes)
+            B.agzo_extract_subspace(ctx, layers, 3, 3)
+            assert B.agzo_poll(ctx) == B.AGZO_OK
+        for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
+            Vo = O.extract_subspace(X, r, 3, 3, i)
+            assert projector_distance(to_host(devs[i][1]), Vo) <= 1e-3
+
+
+def test_extract_rank_deficient_panel_is_reported():
+    rng = np.random.default_rng(0)
+    m, d_in, r = 256, 128, 4
+    X = (np.outer(rng.standard_normal(m), rng.standard_normal(d_in))
+         + np.outer(rng.standard_normal(m), rng.standard_normal(d_in))).astype(np.float32)
+    Vg, st = _run_extract(X, r, 2, seed=3, layer_id=0, path=1, x_bf16=False)
+    assert st == B.AGZO_WARN_RANK_DEFICIENT
+    Vo, info = O.extract_subspace(X, r, 2, 3, 0, return_info=True)
+    assert info["deficient"]
+    assert np.all(Vg[2:] == 0.0) and np.all(Vo[2:] == 0.0)
+    assert projector_distance(Vg[:2], Vo[:2]) <= 1e-3
+
+
+def test_empty_layer_list_and_argument_errors():
+    V = torch.zeros(4, 64, device=DEV)
+    W = torch.zeros(32, 64, device=DEV, dtype=torch.bfloat16)
+    X = torch.zeros(16, 64, device=DEV, dtype=torch.bfloat16)
+    good = B.make_layer(W=W, X=X, V=V, r=4, layer_id=0)
+    with Ctx([good]) as ctx:
+        L = B.lib()
+        assert L.agzo_perturb(ctx.handle, None, 0, 0, 1e-3, None) == B.AGZO_OK
+        assert L.agzo_extract_subspace(ctx.handle, None, 0, 0, 3, None) == B.AGZO_OK
+        assert L.agzo_perturb(ctx.handle, None, 1, 0, 1e-3, None) == B.AGZO_ERR_INVALID_ARG
+
+        def status(fn, layer, *args):
+            return fn(ctx.handle, B.layer_array([layer]), 1, *args)
+
+        bad_r = B.make_layer(W=W, X=X, V=V, r=4, layer_id=0); bad_r.r = 65
+        assert status(L.agzo_perturb, bad_r, 0, 1e-3, None) == B.AGZO_ERR_INVALID_ARG
+        r_gt_m = B.make_layer(W=W, X=X[:2], V=V, r=4, layer_id=0)
+        assert status(L.agzo_extract_subspace, r_gt_m, 0, 3, None) == B.AGZO_ERR_INVALID_ARG
+        no_x = B.make_layer(W=W, V=V, r=4, layer_id=0)
+        assert status(L.agzo_extract_subspace, no_x, 0, 3, None) == B.AGZO_ERR_INVALID_ARG
+        no_w = B.make_layer(X=X, V=V, r=4, layer_id=0)
+        assert status(L.agzo_perturb, no_w, 0, 1e-3, None) == B.AGZO_ERR_INVALID_ARG
+        assert status(L.agzo_extract_subspace, good, 0, 17, None) == B.AGZO_ERR_INVALID_ARG
+        bad_dt = B.make_layer(W=W, X=X, V=V, r=4, layer_id=0); bad_dt.w_dtype = 5
+        assert status(L.agzo_perturb, bad_dt, 0, 1e-3, None) == B.AGZO_ERR_UNSUPPORTED
+        pair_bf16 = B.make_layer(W=W, W16=W, X=X, V=V, r=4, layer_id=0)
+        assert status(L.agzo_perturb, pair_bf16, 0, 1e-3, None) == B.AGZO_ERR_UNSUPPORTED
+        assert L.agzo_update(ctx.handle, B.layer_array([good]), 1, 0, 1e-3, None, None) == B.AGZO_ERR_INVALID_ARG
+        # a workspace that is too small for the layers is refused, nothing is launched
+    small = B.Context(0, 4096)
+    big = B.make_layer(X=torch.zeros(4096, 64, device=DEV), V=V, r=4, layer_id=0)
+    assert B.lib().agzo_extract_subspace(small.handle, B.layer_array([big]), 1, 0, 3, None) == B.AGZO_ERR_WORKSPACE
+    B.agzo_destroy(small)
+    assert bool((W == 0).all())
