@@ -99,10 +99,11 @@ typedef struct agzo_params {
 } agzo_params;
 
 /* Loss callback of agzo_step: run the model's forward on `stream` with the weights as they
- * are now and leave the scalar loss (fp32) at d_loss (device).  phase: 0 = unperturbed
+ * are now and leave the scalar loss at d_loss (device, double: g is a difference of two
+ * nearly equal losses, so an fp32 loss would cap its accuracy near 1e-3 relative).  phase: 0 = unperturbed
  * forward, during or after which the X buffers of the descriptors must have been filled
  * (Algorithm 2, step 1), 1 = at W + mu*Delta, 2 = at W - mu*Delta.  Return 0 on success. */
-typedef int (*agzo_loss_fn)(void* user, void* stream, int phase, float* d_loss);
+typedef int (*agzo_loss_fn)(void* user, void* stream, int phase, double* d_loss);
 
 /* ---------------------------------------------------------------- context and workspace */
 
@@ -165,7 +166,7 @@ agzo_status agzo_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64
  * mode 0: *d_ghat = (*d_f_plus - *d_f_other) / (2 eps)   (f_other = f at W - eps*Delta)
  * mode 1: *d_ghat = (*d_f_plus - *d_f_other) / eps       (f_other = f0)
  * evaluated in double and rounded to fp32.                                               */
-agzo_status agzo_ghat(agzo_ctx* ctx, const float* d_f_plus, const float* d_f_other,
+agzo_status agzo_ghat(agzo_ctx* ctx, const double* d_f_plus, const double* d_f_other,
                       float eps, int mode, float* d_ghat, void* stream);
 
 /* Step 3 of Algorithm 2 as one pass: W_l <- W_l + c * R_l A_l^T with
@@ -179,11 +180,12 @@ agzo_status agzo_restore_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n
 
 /* One AGZO iteration (Algorithm 2): loss(phase 0) -> extract -> perturb(+eps) ->
  * loss(phase 1) -> [mode 0: perturb(-2 eps) -> loss(phase 2)] -> ghat -> restore_update.
- * d_out3 (device, 3 floats) receives f_plus, f_other (f_minus or f0) and g.  If the
- * callback fails, the outstanding perturbation is removed before ERR_CALLBACK returns.   */
+ * d_losses2 (device, 2 doubles) receives f_plus and f_other (f_minus or f0), d_ghat (device,
+ * 1 float) receives g.  If the callback fails, the outstanding perturbation is removed
+ * before ERR_CALLBACK returns.                                                           */
 agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n,
                       const agzo_params* h_params, agzo_loss_fn loss, void* user,
-                      float* d_out3, void* stream);
+                      double* d_losses2, float* d_ghat, void* stream);
 
 /* Second case of Eq. (agzo-perturb), for parameters that are not matrices of a linear
  * layer: w <- w + scale * u with u ~ N(0, I) from (seed, layer_id, tag 2), n_elems

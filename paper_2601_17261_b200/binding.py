@@ -89,7 +89,7 @@ def lib() -> C.CDLL:
         "agzo_update": (i32, [vp, LP, i32, u64, f32, vp, vp]),
         "agzo_ghat": (i32, [vp, vp, vp, f32, i32, vp, vp]),
         "agzo_restore_update": (i32, [vp, LP, i32, u64, f32, f32, i32, vp, vp]),
-        "agzo_step": (i32, [vp, LP, i32, C.POINTER(agzo_params), LOSS_FN, vp, vp, vp]),
+        "agzo_step": (i32, [vp, LP, i32, C.POINTER(agzo_params), LOSS_FN, vp, vp, vp, vp]),
         "agzo_perturb_dense": (i32, [vp, vp, i64, i32, u64, u32, f32, vp, vp]),
         "agzo_debug_philox": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_debug_gaussian": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
@@ -236,6 +236,8 @@ def agzo_update(ctx: Context, layers, seed: int, lr: float, d_ghat: torch.Tensor
 
 def agzo_ghat(ctx: Context, d_f_plus: torch.Tensor, d_f_other: torch.Tensor, eps: float, mode: int,
               d_ghat: torch.Tensor, stream=None) -> None:
+    if d_f_plus.dtype != torch.float64 or d_f_other.dtype != torch.float64:
+        raise TypeError("losses are float64 device scalars")
     _check(lib().agzo_ghat(ctx.handle, d_f_plus.data_ptr(), d_f_other.data_ptr(), eps, mode,
                            d_ghat.data_ptr(), _stream_ptr(stream)), "agzo_ghat")
 
@@ -248,24 +250,28 @@ def agzo_restore_update(ctx: Context, layers, seed: int, eps: float, lr: float, 
 
 
 def agzo_step(ctx: Context, layers, *, seed: int, eps: float, lr: float, K: int, mode: int,
-              loss_fn, d_out3: torch.Tensor, stream=None, arr=None) -> None:
-    """loss_fn(phase:int, d_loss_ptr:int, stream_ptr:int) -> None writes an fp32 scalar at
-    d_loss_ptr on the stream; exceptions become AGZO_ERR_CALLBACK."""
+              loss_fn, d_losses2: torch.Tensor, d_ghat: torch.Tensor, stream=None,
+              arr=None) -> None:
+    """loss_fn(phase:int, slot:int, stream_ptr:int) -> None leaves the float64 loss in
+    d_losses2[slot] on the stream; exceptions become AGZO_ERR_CALLBACK."""
+    if d_losses2.dtype != torch.float64 or d_losses2.numel() < 2 or d_ghat.dtype != torch.float32:
+        raise TypeError("d_losses2 is 2 float64, d_ghat 1 float32 (device)")
+    base = d_losses2.data_ptr()
     arr = arr if arr is not None else layer_array(layers)
     p = agzo_params(seed, eps, lr, K, mode)
     err: List[BaseException] = []
 
     def tramp(user, stream_ptr, phase, d_loss):
         try:
-            loss_fn(int(phase), int(d_loss), int(stream_ptr or 0))
+            loss_fn(int(phase), (int(d_loss) - base) // 8, int(stream_ptr or 0))
             return 0
         except BaseException as e:  # noqa: BLE001 - must not unwind through C
             err.append(e)
             return 1
 
     cb = LOSS_FN(tramp)
-    st = lib().agzo_step(ctx.handle, arr, len(layers), C.byref(p), cb, None, d_out3.data_ptr(),
-                         _stream_ptr(stream))
+    st = lib().agzo_step(ctx.handle, arr, len(layers), C.byref(p), cb, None, d_losses2.data_ptr(),
+                         d_ghat.data_ptr(), _stream_ptr(stream))
     if st == AGZO_ERR_CALLBACK and err:
         raise AgzoError(st, f"agzo_step (callback raised {err[0]!r})")
     _check(st, "agzo_step")

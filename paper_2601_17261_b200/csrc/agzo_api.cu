@@ -487,7 +487,7 @@ agzo_status agzo_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64
   return rmw_pass(ctx, h_layers, n, seed, 0.f, dev_coef(ctx), true, s);
 }
 
-agzo_status agzo_ghat(agzo_ctx* ctx, const float* d_f_plus, const float* d_f_other, float eps,
+agzo_status agzo_ghat(agzo_ctx* ctx, const double* d_f_plus, const double* d_f_other, float eps,
                       int mode, float* d_ghat, void* stream) {
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
@@ -515,10 +515,11 @@ agzo_status agzo_restore_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n
 }
 
 agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n, const agzo_params* p,
-                      agzo_loss_fn loss, void* user, float* d_out3, void* stream) {
+                      agzo_loss_fn loss, void* user, double* d_losses2, float* d_ghat,
+                      void* stream) {
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
-  if (!p || !loss || !d_out3 || !(p->eps > 0.f) || (p->mode != 0 && p->mode != 1) || p->K < 0 ||
+  if (!p || !loss || !d_losses2 || !d_ghat || !(p->eps > 0.f) || (p->mode != 0 && p->mode != 1) || p->K < 0 ||
       p->K > 16)
     return AGZO_ERR_INVALID_ARG;
   st = validate(h_layers, n, NEED_RMW | NEED_EXTRACT);
@@ -526,9 +527,9 @@ agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n, const ag
   bool any_pair = false, any_plain = false;
   for (int i = 0; i < n; ++i) (h_layers[i].W16 ? any_pair : any_plain) = true;
   if (any_pair && any_plain) return AGZO_ERR_UNSUPPORTED;
-  float* d_fplus = d_out3;
-  float* d_fother = d_out3 + 1;
-  float* d_g = d_out3 + 2;
+  double* d_fplus = d_losses2;
+  double* d_fother = d_losses2 + 1;
+  float* d_g = d_ghat;
 
   // step 1: unperturbed forward (fills X), then Algorithm 1 per layer
   if (loss(user, stream, 0, d_fother) != 0) return AGZO_ERR_CALLBACK;

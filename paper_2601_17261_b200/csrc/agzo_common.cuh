@@ -114,7 +114,7 @@ cudaError_t launch_rmw(const DevLayer* d_layers, const int* d_tile_start, int n_
                        int sm_count, cudaStream_t s);
 cudaError_t launch_dense(void* w, long long n, int dtype, uint64_t seed, uint32_t layer_id,
                          float scale, const float* d_scale, cudaStream_t s);
-cudaError_t launch_ghat(const float* fp, const float* fo, float eps, int mode, float* g,
+cudaError_t launch_ghat(const double* fp, const double* fo, float eps, int mode, float* g,
                         cudaStream_t s);
 cudaError_t launch_coef(const float* g, float eps, float lr, int kind, float* d_coef,
                         cudaStream_t s);

@@ -432,11 +432,11 @@ cudaError_t launch_dense(void* w, long long n, int dtype, uint64_t seed, uint32_
 }
 
 // ------------------------------------------------------------------ scalars (Algorithm 2, step 3)
-__global__ void ghat_kernel(const float* fp, const float* fo, float eps, int mode, float* g) {
-  const double d = (double)*fp - (double)*fo;
+__global__ void ghat_kernel(const double* fp, const double* fo, float eps, int mode, float* g) {
+  const double d = *fp - *fo;
   *g = (float)(mode == 0 ? d / (2.0 * (double)eps) : d / (double)eps);
 }
-cudaError_t launch_ghat(const float* fp, const float* fo, float eps, int mode, float* g, cudaStream_t s) {
+cudaError_t launch_ghat(const double* fp, const double* fo, float eps, int mode, float* g, cudaStream_t s) {
   ghat_kernel<<<1, 1, 0, s>>>(fp, fo, eps, mode, g);
   return cudaGetLastError();
 }
