@@ -1,0 +1,347 @@
+"""Benchmark of the AGZO per-step hot path on synthetic Qwen3-shaped layer sets.
+
+One "step" = Algorithm 1 for every layer (K = 3) + the three in-place passes of a two-point
+AGZO iteration (perturb +eps, flip -2 eps, fused restore-and-update) + the scalar; forward
+passes are the caller's model and are excluded ("step overhead").  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--rank R]
+  python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of
+the same step on its own GPU (the path has no exchange step; weights are replicated in
+zeroth-order data parallelism and every rank applies the same seeded perturbation).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2601_17261_b200 import workloads as WL  # noqa: E402
+
+K_POWER = 3
+EPS = 1e-3
+LR = 1e-6
+METRIC = "agzo_step_overhead_ms"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "200", "-i", str(device_index)], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(",") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[5:9]):
+                if v.strip().lower() == "active":
+                    reasons.add(nm)
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+            out["sm_max_mhz"] = float(max(mx))
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- workload
+def build_layer_set(cfg: WL.LayerSetConfig, rank: int, device, seed: int = 1000):
+    """Resident tensors of one layer set: bf16 W and X per layer (torch device generators,
+    same recipe as the host generators the parity tests use), fp32 V."""
+    from paper_2601_17261_b200 import binding as B
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    Ws, Xs, Vs, layers = [], [], [], []
+    for i, (name, d_in, d_out) in enumerate(cfg.layers()):
+        W = WL.device_weights(d_out, d_in, cfg.w_std, gen, device)
+        X = WL.device_planted_activations(cfg.m, d_in, cfg.planted_rank, gen, device)
+        V = torch.zeros(rank, d_in, dtype=torch.float32, device=device)
+        Ws.append(W); Xs.append(X); Vs.append(V)
+        layers.append(B.make_layer(W=W, X=X, V=V, r=rank, layer_id=i))
+    return Ws, Xs, Vs, layers
+
+
+def algorithmic_work(cfg: WL.LayerSetConfig, rank: int):
+    n_w = cfg.n_params()
+    x_elems = cfg.x_elems()
+    rmw_bytes_pass = 4 * n_w + sum(4 * rank * di for (_, di, _) in cfg.layers())
+    extract_bytes = (K_POWER + 1) * 2 * x_elems          # X read once per product pair (fused)
+    extract_bytes_unfused = (2 * K_POWER + 1) * 2 * x_elems
+    extract_flops = sum((2 * K_POWER + 1) * 2 * cfg.m * di * rank + (K_POWER + 1) * 2 * di * rank * rank
+                        for (_, di, _) in cfg.layers())
+    return {"rmw_bytes_per_pass": rmw_bytes_pass, "extract_bytes_fused": extract_bytes,
+            "extract_bytes_unfused": extract_bytes_unfused, "extract_flops": extract_flops,
+            "x_bytes": 2 * x_elems, "w_bytes": 2 * n_w}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_block_seconds(cfg: WL.LayerSetConfig, rank: int, X_host, W_host, seed: int = 0):
+    """The oracle, as it stands, on block 0 (7 layers): Algorithm 1 + the three passes."""
+    from oracle import agzo_oracle as O
+    t0 = time.perf_counter()
+    for i, (X, W) in enumerate(zip(X_host, W_host)):
+        V = O.extract_subspace(X, rank, K_POWER, seed, i)
+        W1 = O.apply_direction(W, V, seed, i, np.float32(EPS), "bf16")
+        W2 = O.apply_direction(W1, V, seed, i, np.float32(-2 * EPS), "bf16")
+        g = O.ghat_two_point(1.0, 0.999, EPS)
+        O.apply_direction(W2, V, seed, i, O.update_coefficient(EPS, LR, g, 0), "bf16")
+    return time.perf_counter() - t0
+
+
+def host_block(cfg: WL.LayerSetConfig, n_layers: int = 7, seed: int = 1000):
+    """First layers of block 0 generated on the host with the numpy recipe (bf16 values as float32)."""
+    Xs, Ws = [], []
+    for i, (name, d_in, d_out) in enumerate(cfg.block[:n_layers]):
+        Xs.append(WL.planted_activations(cfg.m, d_in, cfg.planted_rank, seed + i, bf16=True))
+        Ws.append(WL.gaussian_weights(d_out, d_in, cfg.w_std, seed + i, bf16=True))
+    return Xs, Ws
+
+
+def run_reference(args, cfg, rank_r):
+    """--impl reference: the CPU oracle on the host cores; a step = block 0 of the layer set,
+    extrapolated to all blocks (every block has the same shapes)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    cores = os.cpu_count() or 1
+    Xs, Ws = host_block(cfg)
+    times = []
+    for it in range(args.warmup + args.steps):
+        t = oracle_block_seconds(cfg, rank_r, Xs, Ws, seed=it)
+        if it >= args.warmup:
+            times.append(t)
+    ms = float(np.mean(times)) * 1e3 * cfg.n_blocks
+    sample = f"block 0 (7 of {7 * cfg.n_blocks} layers) per step, time x{cfg.n_blocks}"
+    line = {"metric": METRIC, "value": ms, "unit": "ms", "impl": "reference", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}, r={rank_r}, K={K_POWER}, m={cfg.m}", "sample": sample},
+            "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": ms, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------- main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="agzo", choices=["agzo", "reference"])
+    ap.add_argument("--workload", default=WL.QWEN3_8B.name, choices=sorted(WL.LAYER_SETS))
+    ap.add_argument("--rank", type=int, default=16)
+    ap.add_argument("--extract-path", type=int, default=0)
+    ap.add_argument("--wave-mb", type=int, default=-1)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    cfg = WL.LAYER_SETS[args.workload]
+    r = args.rank
+    if args.impl == "reference":
+        return run_reference(args, cfg, r)
+
+    from paper_2601_17261_b200 import binding as B
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the AGZO path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()   # fails loudly when the CUDA library is missing
+
+    Ws, Xs, Vs, layers = build_layer_set(cfg, r, dev)
+    arr = B.layer_array(layers)
+    ctx = B.agzo_create(layers, local)
+    B.agzo_set_option(ctx, "extract_path", args.extract_path)
+    if args.wave_mb >= 0:
+        B.agzo_set_option(ctx, "wave_bytes", args.wave_mb << 20)
+    work = algorithmic_work(cfg, r)
+    losses = torch.tensor([1.0, 0.999], dtype=torch.float64, device=dev)
+    ghat = torch.zeros(1, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(seed: int):
+        B.agzo_extract_subspace(ctx, layers, seed, K_POWER, arr=arr)
+        B.agzo_perturb(ctx, layers, seed, EPS, arr=arr)
+        B.agzo_perturb(ctx, layers, seed, -2 * EPS, arr=arr)
+        B.agzo_ghat(ctx, losses[0:1], losses[1:2], EPS, 0, ghat)
+        B.agzo_restore_update(ctx, layers, seed, EPS, LR, 0, ghat, arr=arr)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, n, first_seed):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(n):
+            fn(first_seed + i)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1) / n
+        if dist is not None:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t)
+        return ms
+
+    # ---- warm-up, then the timed region with the dominant kernel class bracketed by events
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if B.agzo_poll(ctx) not in (B.AGZO_OK,):
+        raise SystemExit("device status not ok after warm-up")
+    tc_used = args.extract_path != 1 and False
+    dom_class = B.KC_XT_T
+    B.agzo_set_option(ctx, "time_kernel_class", dom_class)
+    B.agzo_read_counters(ctx)
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms_step = timed(step, args.steps, 100)
+    clocks = sampler.stop() if sampler else {}
+    dom_ms, dom_n, launches = B.agzo_read_counters(ctx)
+    B.agzo_set_option(ctx, "time_kernel_class", 0)
+
+    # ---- per-phase timings (outside the timed region), same kernels
+    def phase_ms(fn, n=3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(n):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    ms_extract = phase_ms(lambda i: B.agzo_extract_subspace(ctx, layers, 200 + i, K_POWER, arr=arr), 2)
+    ms_perturb = phase_ms(lambda i: B.agzo_perturb(ctx, layers, 300 + i, EPS if i % 2 == 0 else -EPS, arr=arr), 4)
+    ms_update = phase_ms(lambda i: B.agzo_restore_update(ctx, layers, 400 + i, EPS, LR, 0, ghat, arr=arr), 4)
+
+    # ---- end to end: the step's activations arrive from pinned host memory, ghat goes back
+    e2e = None
+    if not args.no_e2e:
+        blk = len(cfg.block)
+        pinned = [torch.empty_like(Xs[j], device="cpu").pin_memory() for j in range(blk)]
+        for j in range(blk):
+            pinned[j].copy_(Xs[j])
+        g_host = torch.empty(1, dtype=torch.float32).pin_memory()
+        h2d = sum(x.numel() * 2 for x in Xs)
+
+        def e2e_step(seed):
+            for i, X in enumerate(Xs):
+                X.copy_(pinned[i % blk], non_blocking=True)
+            step(seed)
+            g_host.copy_(ghat, non_blocking=True)
+
+        e2e_step(0)
+        ms_e2e = timed(e2e_step, max(1, min(args.steps, 3)), 500)
+        e2e = {"value": ms_e2e, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
+               "note": "X of every layer copied from pinned host memory each step (one block's "
+                       "pinned buffers reused for all blocks), ghat copied back"}
+
+    status = B.agzo_poll(ctx)
+    peak, peak_kind = measured_peaks()
+    x_bytes_per_launch = work["x_bytes"] * (K_POWER + 1) / max(dom_n / max(args.steps, 1), 1)
+    dom_avg_ms = dom_ms / max(dom_n, 1)
+    achieved = x_bytes_per_launch / (dom_avg_ms * 1e-3) / 1e9 if dom_n else None
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": ms_step, "unit": "ms", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic",
+            "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: {len(layers)} layers, {cfg.n_params() / 1e9:.3f} G weights, "
+                                   f"m={cfg.m} tokens, r={r}, K={K_POWER}, eps={EPS}, two-point",
+                       "l2": "inputs larger than L2 (weights %.1f GB + activations %.1f GB per step)"
+                             % (work["w_bytes"] / 1e9, work["x_bytes"] / 1e9),
+                       "replicas": world, "device_status": B.status_string(status)},
+            "phases_ms": {"extract": ms_extract, "perturb": ms_perturb, "restore_update": ms_update},
+            "rmw": {"GBps_perturb": work["rmw_bytes_per_pass"] / ms_perturb / 1e6,
+                    "GBps_restore_update": work["rmw_bytes_per_pass"] / ms_update / 1e6,
+                    "frac_of_%s_hbm" % peak_kind: work["rmw_bytes_per_pass"] / ms_perturb / 1e6 / peak,
+                    "frac_of_nominal_8TBps": work["rmw_bytes_per_pass"] / ms_perturb / 1e6 / 8000.0},
+            "extract": {"TFLOPs_algorithmic": work["extract_flops"] / ms_extract / 1e9,
+                        "GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6},
+            "roofline": {"kernel": "xt_t (Y = X^T T)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+                         "peak_kind": peak_kind, "traffic": None,
+                         "launches": dom_n, "avg_ms": dom_avg_ms},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if e2e:
+            line["e2e"] = e2e
+        if not args.no_cpu_baseline and world == 1:
+            Xh, Wh = host_block(cfg, 1)
+            # one layer of block 0 keeps the CPU leg within tens of seconds
+            t = oracle_block_seconds(cfg, r, Xh, Wh)
+            scale = sum(di * (cfg.m + do) for (_, di, do) in cfg.block) / (cfg.block[0][1] * (cfg.m + cfg.block[0][2]))
+            line["cpu_baseline"] = {"value": t * 1e3 * scale * cfg.n_blocks, "unit": "ms",
+                                    "cores": os.cpu_count(), "kind": "oracle",
+                                    "sample": f"layer 0.q of {len(layers)} layers timed ({t:.2f} s), scaled by "
+                                              f"elements touched to the whole set (x{scale * cfg.n_blocks:.1f})"}
+        print(json.dumps(line))
+    B.agzo_destroy(ctx)
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -120,8 +120,28 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
 
 /* Options: "extract_path" 0 = automatic, 1 = CUDA-core fp32 kernels only, 2 = require the
  * tensor-core kernels (UNSUPPORTED at call time if a layer cannot use them);
- * "wave_bytes" = activation bytes grouped into one launch wave of extraction.            */
+ * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
+ * "time_kernel_class" = one agzo_kernel_class whose launches get a CUDA event pair on the
+ * caller's stream (0 = none), read back by agzo_read_counters.                           */
 agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value);
+
+typedef enum agzo_kernel_class {
+  AGZO_KC_NONE = 0,
+  AGZO_KC_RMW = 1,        /* the in-place low-rank pass                                    */
+  AGZO_KC_XT_T = 2,       /* Y = X^T T, CUDA-core kernel                                   */
+  AGZO_KC_X_Q = 3,        /* T = X Q, CUDA-core kernel                                     */
+  AGZO_KC_PANEL_QR = 4,   /* the three kernels of qr(Y) as one unit                        */
+  AGZO_KC_TC_XT_T = 5,    /* Y = X^T T, tensor-core kernel                                 */
+  AGZO_KC_TC_X_Q = 6,     /* T = X Q, tensor-core kernel                                   */
+  AGZO_KC_OMEGA = 7       /* Gaussian test matrix fill                                     */
+} agzo_kernel_class;
+
+/* Measurement aid.  Waits for the timed launches recorded since the last read, then returns
+ * their summed device time in milliseconds, how many there were, and the number of kernel
+ * launches of every class the context has issued since the last read; all three counters
+ * are reset.  Any output pointer may be NULL.  Synchronises with the timed events only.   */
+agzo_status agzo_read_counters(agzo_ctx* ctx, double* h_ms, int64_t* h_timed_launches,
+                               int64_t* h_total_launches);
 
 /* Waits for the stream work of this context issued so far on `stream` and returns the
  * device status word: AGZO_OK, AGZO_WARN_RANK_DEFICIENT or AGZO_ERR_TIMEOUT; the word is

@@ -30,8 +30,9 @@ EXPORTS = [
     "agzo_workspace_bytes", "agzo_create", "agzo_destroy", "agzo_set_option", "agzo_poll",
     "agzo_status_string", "agzo_last_cuda_error", "agzo_extract_subspace", "agzo_perturb",
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
-    "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian",
+    "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
 ]
+KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA = 1, 2, 3, 4, 5, 6, 7
 
 
 class agzo_layer(C.Structure):
@@ -93,6 +94,7 @@ def lib() -> C.CDLL:
         "agzo_perturb_dense": (i32, [vp, vp, i64, i32, u64, u32, f32, vp, vp]),
         "agzo_debug_philox": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_debug_gaussian": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
+        "agzo_read_counters": (i32, [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -203,6 +205,14 @@ def agzo_destroy(ctx: Context) -> None:
 
 def agzo_set_option(ctx: Context, name: str, value: int) -> None:
     _check(lib().agzo_set_option(ctx.handle, name.encode(), int(value)), "agzo_set_option")
+
+
+def agzo_read_counters(ctx: Context):
+    """(summed ms of the timed kernel class, its launches, launches of every class)."""
+    ms, nt, na = C.c_double(0), C.c_int64(0), C.c_int64(0)
+    _check(lib().agzo_read_counters(ctx.handle, C.byref(ms), C.byref(nt), C.byref(na)),
+           "agzo_read_counters")
+    return ms.value, nt.value, na.value
 
 
 def agzo_poll(ctx: Context, stream=None) -> int:

@@ -52,6 +52,11 @@ struct agzo_ctx {
   cudaEvent_t stage_ev;
   bool stage_pending;
   TcState tc;
+  // measurement aid: event pairs around the launches of one kernel class
+  int time_class;
+  std::vector<cudaEvent_t> events;   // pairs: start, stop
+  size_t events_used;
+  int64_t launches;
 };
 
 namespace {
@@ -64,6 +69,31 @@ namespace {
       return AGZO_ERR_CUDA;                        \
     }                                              \
   } while (0)
+
+// Launch bookkeeping: counts every kernel-launching call and, for the class being timed,
+// brackets it with an event pair on the stream.
+struct Timed {
+  agzo_ctx* c;
+  cudaStream_t s;
+  bool on;
+  Timed(agzo_ctx* ctx, int cls, cudaStream_t st, int n_kernels = 1) : c(ctx), s(st), on(false) {
+    c->launches += n_kernels;
+    if (c->time_class != cls) return;
+    if (c->events_used + 2 > c->events.size()) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        c->events.push_back(e);
+      }
+    }
+    on = cudaEventRecord(c->events[c->events_used], s) == cudaSuccess;
+  }
+  ~Timed() {
+    if (!on) return;
+    cudaEventRecord(c->events[c->events_used + 1], s);
+    c->events_used += 2;
+  }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -279,6 +309,7 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   if (n == 0) return AGZO_OK;
   st = prepare(c, L, n, s);
   if (st != AGZO_OK) return st;
+  Timed t(c, AGZO_KC_RMW, s);
   CU(c, launch_rmw(dev_layers(c), dev_tiles(c, n), n, c->plan.total_tiles, c->plan.max_r,
                    c->plan.fast_mode_mask, c->plan.any_slow, seed, coef, d_coef, pair_update,
                    c->sm_count, s));
@@ -342,6 +373,9 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->h_stage_bytes = 0;
   c->stage_pending = false;
   c->stage_ev = nullptr;
+  c->time_class = 0;
+  c->events_used = 0;
+  c->launches = 0;
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->stage_ev, cudaEventDisableTiming);
@@ -362,6 +396,7 @@ agzo_status agzo_destroy(agzo_ctx* ctx) {
   if (ctx->stage_pending) cudaEventSynchronize(ctx->stage_ev);
   if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
   if (ctx->stage_ev) cudaEventDestroy(ctx->stage_ev);
+  for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   ctx->magic = 0;
   delete ctx;
   return AGZO_OK;
@@ -376,10 +411,32 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
   } else if (std::strcmp(name, "wave_bytes") == 0) {
     if (value < 0) return AGZO_ERR_INVALID_ARG;
     ctx->wave_bytes = value;
+  } else if (std::strcmp(name, "time_kernel_class") == 0) {
+    if (value < 0 || value > 7) return AGZO_ERR_INVALID_ARG;
+    ctx->time_class = (int)value;
+    return AGZO_OK;
   } else {
     return AGZO_ERR_INVALID_ARG;
   }
   ctx->cached_valid = false;   // the plan depends on the options
+  return AGZO_OK;
+}
+
+agzo_status agzo_read_counters(agzo_ctx* ctx, double* h_ms, int64_t* h_timed, int64_t* h_total) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  double ms = 0.0;
+  for (size_t i = 0; i + 1 < ctx->events_used; i += 2) {
+    CU(ctx, cudaEventSynchronize(ctx->events[i + 1]));
+    float t = 0.f;
+    CU(ctx, cudaEventElapsedTime(&t, ctx->events[i], ctx->events[i + 1]));
+    ms += (double)t;
+  }
+  if (h_ms) *h_ms = ms;
+  if (h_timed) *h_timed = (int64_t)(ctx->events_used / 2);
+  if (h_total) *h_total = ctx->launches;
+  ctx->events_used = 0;
+  ctx->launches = 0;
   return AGZO_OK;
 }
 
@@ -431,26 +488,30 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
     l0 = l1;
     if (w.max_m == 0) continue;
     DevStatus* dst = dev_status(ctx);
-    if (all_tc) {
-      // tensor-core products; the panel factorisation is shared
-      CU(ctx, tc_fill_omega(ctx->tc, w, P.dev.data(), seed, s));
-      CU(ctx, tc_xt_t(ctx->tc, w, P.dev.data(), dst, s));
-      for (int k = 0; k < K; ++k) {
-        CU(ctx, launch_panel_qr(w, dst, s));
-        CU(ctx, tc_x_q(ctx->tc, w, P.dev.data(), dst, s));
-        CU(ctx, tc_xt_t(ctx->tc, w, P.dev.data(), dst, s));
-      }
-      CU(ctx, launch_panel_qr(w, dst, s));
-    } else {
-      CU(ctx, launch_fill_omega(w, seed, s));
-      CU(ctx, launch_xt_t(w, s));
-      for (int k = 0; k < K; ++k) {
-        CU(ctx, launch_panel_qr(w, dst, s));
-        CU(ctx, launch_x_q(w, s));
-        CU(ctx, launch_xt_t(w, s));
-      }
-      CU(ctx, launch_panel_qr(w, dst, s));
+    auto panel_qr = [&]() -> cudaError_t {
+      Timed t(ctx, AGZO_KC_PANEL_QR, s, 3);
+      return launch_panel_qr(w, dst, s);
+    };
+    auto omega = [&]() -> cudaError_t {
+      Timed t(ctx, AGZO_KC_OMEGA, s);
+      return all_tc ? tc_fill_omega(ctx->tc, w, P.dev.data(), seed, s) : launch_fill_omega(w, seed, s);
+    };
+    auto xt_t = [&]() -> cudaError_t {       // Y <- H T
+      Timed t(ctx, all_tc ? AGZO_KC_TC_XT_T : AGZO_KC_XT_T, s);
+      return all_tc ? tc_xt_t(ctx->tc, w, P.dev.data(), dst, s) : launch_xt_t(w, s);
+    };
+    auto x_q = [&]() -> cudaError_t {        // T <- H^T Q
+      Timed t(ctx, all_tc ? AGZO_KC_TC_X_Q : AGZO_KC_X_Q, s);
+      return all_tc ? tc_x_q(ctx->tc, w, P.dev.data(), dst, s) : launch_x_q(w, s);
+    };
+    CU(ctx, omega());                        // Omega
+    CU(ctx, xt_t());                         // Y <- H Omega
+    for (int k = 0; k < K; ++k) {
+      CU(ctx, panel_qr());                   // Q <- qr(Y)
+      CU(ctx, x_q());
+      CU(ctx, xt_t());                       // Y <- H (H^T Q)
     }
+    CU(ctx, panel_qr());                     // A <- qr(Y)
   }
   return AGZO_OK;
 }
@@ -483,6 +544,7 @@ agzo_status agzo_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64
   st = validate(h_layers, n, NEED_RMW);
   if (st != AGZO_OK) return st;
   if (n == 0) return AGZO_OK;
+  ctx->launches += 1;
   CU(ctx, launch_coef(d_ghat, 0.f, lr, 2, dev_coef(ctx), s));
   return rmw_pass(ctx, h_layers, n, seed, 0.f, dev_coef(ctx), true, s);
 }
@@ -493,6 +555,7 @@ agzo_status agzo_ghat(agzo_ctx* ctx, const double* d_f_plus, const double* d_f_o
   if (st != AGZO_OK) return st;
   if (!d_f_plus || !d_f_other || !d_ghat || !(eps > 0.f) || (mode != 0 && mode != 1))
     return AGZO_ERR_INVALID_ARG;
+  ctx->launches += 1;
   CU(ctx, launch_ghat(d_f_plus, d_f_other, eps, mode, d_ghat, static_cast<cudaStream_t>(stream)));
   return AGZO_OK;
 }
@@ -510,6 +573,7 @@ agzo_status agzo_restore_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n
   for (int i = 0; i < n; ++i) (h_layers[i].W16 ? any_pair : any_plain) = true;
   if (any_pair && any_plain) return AGZO_ERR_UNSUPPORTED;
   // a pair's master was never perturbed: only the update term applies to it
+  ctx->launches += 1;
   CU(ctx, launch_coef(d_ghat, eps, lr, any_pair ? 2 : mode, dev_coef(ctx), s));
   return rmw_pass(ctx, h_layers, n, seed, 0.f, dev_coef(ctx), true, s);
 }
