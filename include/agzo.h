@@ -215,6 +215,35 @@ agzo_status agzo_perturb_dense(agzo_ctx* ctx, void* w, int64_t n_elems, int dtyp
                                uint64_t seed, uint32_t layer_id, float scale,
                                const float* d_scale, void* stream);
 
+/* ---------------------------------------------------------------- allocation-free variant */
+
+/* (No counterpart in the paper: this entry point exists for callers, not for the method.)
+ * Algorithm 1 for ONE layer without a context or a workspace: the same kernels as
+ * agzo_extract_subspace's CUDA-core path, with their scratch in a fixed 4 MiB array that is
+ * part of the library image on every GPU that loads it.  It is meant for callers that cannot
+ * allocate device memory where they need a subspace -- a forward hook that runs while
+ * another framework owns (or has frozen) the allocator, a callback in which an allocation
+ * would synchronise the device, a job whose memory is fixed up front.  X and V are still
+ * the caller's.  The call itself performs no cudaMalloc / cudaFree and calls no library
+ * routine that allocates.
+ *   X [m][ldx] (x_dtype), V [r][ldv] fp32 out, d_rank_deficient: optional device int32 that
+ *   receives 1 when a panel column was zeroed (see AGZO_WARN_RANK_DEFICIENT), else 0.
+ * Limit: the scratch of the problem must fit the array,
+ *   512 + 4 m r + 4 slabs r d_in + 4 r d_in + 8 ceil(d_in/128) r^2 + 8 r^2  <=  4 MiB
+ *   (each term rounded up to 256 bytes; slabs = ceil(m / max(256, ceil32(ceil(m/32)))));
+ *   for example m = 4096, d_in = 2048, r = 16 fits, m = 16384, d_in = 4096, r = 16 does not.
+ *   Larger problems are refused with AGZO_ERR_WORKSPACE and nothing is launched.
+ * Uses the CURRENT CUDA device.  The first call on each device looks up the array's device
+ * address (cudaGetSymbolAddress); make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's contents (the
+ * call clears what must start clean).  Two calls whose GPU work can overlap -- different
+ * streams without an ordering between them, or different host threads -- race on it: order
+ * them on one stream or with events.  Other errors: INVALID_ARG, UNSUPPORTED, CUDA.        */
+agzo_status agzo_extract_subspace_static(const void* X, int64_t ldx, int32_t x_dtype, int32_t m,
+                                         int32_t d_in, int32_t r, int32_t K, uint64_t seed,
+                                         uint32_t layer_id, float* V, int64_t ldv,
+                                         int32_t* d_rank_deficient, void* stream);
+
 /* ---------------------------------------------------------------- test exports */
 
 /* Raw Philox words / normals of elements first .. first+n-1 of stream (seed, layer_id, tag)

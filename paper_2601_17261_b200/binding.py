@@ -31,6 +31,7 @@ EXPORTS = [
     "agzo_status_string", "agzo_last_cuda_error", "agzo_extract_subspace", "agzo_perturb",
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
+    "agzo_extract_subspace_static",
 ]
 KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA = 1, 2, 3, 4, 5, 6, 7
 
@@ -95,6 +96,8 @@ def lib() -> C.CDLL:
         "agzo_debug_philox": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_debug_gaussian": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_read_counters": (i32, [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)]),
+        "agzo_extract_subspace_static": (i32, [vp, i64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                               C.c_int32, u64, u32, vp, i64, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -223,6 +226,21 @@ def agzo_extract_subspace(ctx: Context, layers, seed: int, K: int, stream=None, 
     arr = arr if arr is not None else layer_array(layers)
     _check(lib().agzo_extract_subspace(ctx.handle, arr, len(layers), seed, K, _stream_ptr(stream)),
            "agzo_extract_subspace")
+
+
+def agzo_extract_subspace_static(X: torch.Tensor, V: torch.Tensor, r: int, K: int, seed: int,
+                                 layer_id: int, d_rank_deficient: Optional[torch.Tensor] = None,
+                                 stream=None) -> None:
+    """Algorithm 1 for one layer with the library's built-in scratch: for callers that cannot
+    allocate a workspace (see include/agzo.h).  No context; allocates nothing; uses the current
+    device; calls that can overlap on the GPU must be ordered by the caller."""
+    if X.dim() != 2 or X.stride(1) != 1 or V.dim() != 2 or V.stride(1) != 1 or V.dtype != torch.float32:
+        raise ValueError("X [m][ldx] and V [r][ldv] (fp32) need unit inner strides")
+    flag = d_rank_deficient.data_ptr() if d_rank_deficient is not None else None
+    _check(lib().agzo_extract_subspace_static(X.data_ptr(), X.stride(0), _dtype_code(X), X.shape[0],
+                                              X.shape[1], r, K, seed, layer_id, V.data_ptr(),
+                                              V.stride(0), flag, _stream_ptr(stream)),
+           "agzo_extract_subspace_static")
 
 
 def agzo_perturb(ctx: Context, layers, seed: int, scale: float, stream=None, arr=None) -> None:
