@@ -247,8 +247,8 @@ def main():
     torch.cuda.synchronize()
     if B.agzo_poll(ctx) not in (B.AGZO_OK,):
         raise SystemExit("device status not ok after warm-up")
-    tc_used = args.extract_path != 1 and False
-    dom_class = B.KC_XT_T
+    tc_used = args.extract_path != 1
+    dom_class = B.KC_TC_XT_T if tc_used else B.KC_XT_T
     B.agzo_set_option(ctx, "time_kernel_class", dom_class)
     B.agzo_read_counters(ctx)
     sampler = ClockSampler(local) if rank == 0 else None
@@ -318,7 +318,7 @@ def main():
                     "frac_of_nominal_8TBps": work["rmw_bytes_per_pass"] / ms_perturb / 1e6 / 8000.0},
             "extract": {"TFLOPs_algorithmic": work["extract_flops"] / ms_extract / 1e9,
                         "GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6},
-            "roofline": {"kernel": "xt_t (Y = X^T T)", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": ("tc_xt_t_kernel" if tc_used else "xt_t_kernel") + " (Y = X^T T)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                          "peak_kind": peak_kind, "traffic": None,
                          "launches": dom_n, "avg_ms": dom_avg_ms},

@@ -131,9 +131,19 @@ agzo_status validate(const agzo_layer* L, int n, int need) {
 
 bool has_x(const agzo_layer& a) { return a.X != nullptr && a.m >= 1; }
 
-void slab_shape(const agzo_layer& a, int* slabs, int* slab_rows) {
-  int rows = (a.m + 31) / 32;
-  rows = (rows + 31) / 32 * 32;
+// Token slabs of the X^T T product.  CUDA-core kernels: 32 slabs at most.  Tensor-core
+// kernels: enough (column chunk, slab) CTAs to fill the GPU twice, slabs a multiple of 64 tokens.
+void slab_shape(const agzo_layer& a, bool tc, int* slabs, int* slab_rows) {
+  int rows;
+  if (tc) {
+    const int chunks = (a.d_in + 127) / 128;
+    const int want = (2 * 148 + chunks - 1) / chunks;
+    rows = (a.m + want - 1) / want;
+    rows = (rows + 63) / 64 * 64;
+  } else {
+    rows = (a.m + 31) / 32;
+    rows = (rows + 31) / 32 * 32;
+  }
   if (rows < 256) rows = 256;
   *slab_rows = rows;
   *slabs = (a.m + rows - 1) / rows;
@@ -143,7 +153,7 @@ void slab_shape(const agzo_layer& a, int* slabs, int* slab_rows) {
 size_t layer_scratch(const agzo_layer& a, bool tc) {
   if (!has_x(a)) return 0;
   int slabs, slab_rows;
-  slab_shape(a, &slabs, &slab_rows);
+  slab_shape(a, tc, &slabs, &slab_rows);
   const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
   const size_t gch = (d + 127) / 128;
   size_t b = 0;
@@ -156,13 +166,18 @@ size_t layer_scratch(const agzo_layer& a, bool tc) {
   return b;
 }
 
+constexpr size_t kMapBytes = 512;   // four TMA descriptors per layer
 size_t table_bytes(int n) {
-  return align_up((size_t)n * sizeof(DevLayer)) + align_up((size_t)(n + 1) * sizeof(int));
+  return align_up((size_t)n * sizeof(DevLayer)) + align_up((size_t)(n + 1) * sizeof(int)) +
+         align_up((size_t)n * kMapBytes);
+}
+size_t maps_offset(int n) {
+  return kHeaderBytes + align_up((size_t)n * sizeof(DevLayer)) + align_up((size_t)(n + 1) * sizeof(int));
 }
 
 // Builds the device records.  ws == nullptr: only sizes are computed (scratch_needed).
 agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, int64_t wave_bytes,
-                       int extract_path, Plan* plan, size_t* scratch_needed) {
+                       int extract_path, bool tc_available, Plan* plan, size_t* scratch_needed) {
   plan->dev.assign(n, DevLayer{});
   plan->tile_start.assign(n + 1, 0);
   plan->wave_end.clear();
@@ -214,7 +229,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
     int64_t xbytes = 0;
     int j = i;
     while (j < n && has_x(L[j])) {
-      const bool tc = extract_path != 1 && tc_eligible(L[j]);
+      const bool tc = extract_path != 1 && tc_available && tc_eligible(L[j]);
       const size_t need = layer_scratch(L[j], tc);
       const int64_t xb = (int64_t)L[j].m * L[j].d_in * (L[j].x_dtype == AGZO_BF16 ? 2 : 4);
       if (j > i && (used + need > scratch_cap || xbytes + xb > wave_bytes)) break;
@@ -225,7 +240,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
         DevLayer& D = plan->dev[j];
         const agzo_layer& a = L[j];
         int slabs, slab_rows;
-        slab_shape(a, &slabs, &slab_rows);
+        slab_shape(a, tc, &slabs, &slab_rows);
         const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
         const size_t gch = (d + 127) / 128;
         D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
@@ -234,7 +249,10 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
         D.Y = reinterpret_cast<float*>(p);      p += align_up(r * d * 4);
         D.Gpart = reinterpret_cast<double*>(p); p += align_up(gch * r * r * 8);
         D.M = reinterpret_cast<double*>(p);     p += align_up(r * r * 8);
-        if (tc) tc_carve(a, &D, p);
+        if (tc) {
+          tc_carve(a, &D, p);
+          D.tmaps = ws + maps_offset(n) + (size_t)j * kMapBytes;
+        }
       }
       used += need;
       xbytes += xb;
@@ -265,10 +283,11 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (same_layers(c, L, n)) return AGZO_OK;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
-  agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, c->wave_bytes, c->extract_path, &plan, nullptr);
+  agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, c->wave_bytes, c->extract_path,
+                              c->tc.available, &plan, nullptr);
   if (st != AGZO_OK) return st;
   const size_t lb = align_up((size_t)n * sizeof(DevLayer));
-  const size_t tb = (size_t)(n + 1) * sizeof(int);
+  const size_t tb = align_up((size_t)(n + 1) * sizeof(int)) + (size_t)n * kMapBytes;
   if (c->stage_pending) {
     CU(c, cudaEventSynchronize(c->stage_ev));
     c->stage_pending = false;
@@ -282,7 +301,14 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   }
   if (n > 0) {
     std::memcpy(c->h_stage, plan.dev.data(), (size_t)n * sizeof(DevLayer));
-    std::memcpy(static_cast<char*>(c->h_stage) + lb, plan.tile_start.data(), tb);
+    char* hs = static_cast<char*>(c->h_stage);
+    std::memset(hs + lb, 0, tb);
+    std::memcpy(hs + lb, plan.tile_start.data(), (size_t)(n + 1) * sizeof(int));
+    char* hmaps = hs + lb + align_up((size_t)(n + 1) * sizeof(int));
+    for (int i = 0; i < n; ++i) {
+      if (!plan.dev[i].Qb) continue;
+      if (!tc_encode_maps(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes)) return AGZO_ERR_UNSUPPORTED;
+    }
     CU(c, cudaMemcpyAsync(c->ws + kHeaderBytes, c->h_stage, lb + tb, cudaMemcpyHostToDevice, s));
     CU(c, cudaEventRecord(c->stage_ev, s));
     c->stage_pending = true;
@@ -344,7 +370,7 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   if (st != AGZO_OK) return st;
   Plan plan;
   size_t scratch = 0;
-  st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 0, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 0, true, &plan, &scratch);
   if (st != AGZO_OK) return st;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
   return AGZO_OK;
@@ -464,7 +490,7 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (ctx->extract_path == 2)
     for (int i = 0; i < n; ++i)
-      if (!tc_eligible(h_layers[i])) return AGZO_ERR_UNSUPPORTED;
+      if (!ctx->tc.available || !tc_eligible(h_layers[i])) return AGZO_ERR_UNSUPPORTED;
   st = prepare(ctx, h_layers, n, s);
   if (st != AGZO_OK) return st;
 

@@ -33,8 +33,10 @@ struct alignas(16) DevLayer {
   int gchunks;           // column chunks of the Gram reduction
   int x_vec_ok;          // X rows 16-byte aligned
   // tensor-core path panels (bf16 hi/lo splits), null when unused
-  __nv_bfloat16* Qb;     // [NB][d_in]  rows 0..r-1 hi parts, rows NP..NP+r-1 lo parts
-  __nv_bfloat16* Tb;     // [m][NB]     same split along the columns
+  __nv_bfloat16* Qb;     // [NB][d_in]   rows 0..r-1 hi parts, rows NP..NP+r-1 lo parts, other rows zero
+  __nv_bfloat16* Tb;     // [NB][m_pad]  T transposed, same row split
+  const void* tmaps;     // four 128-byte TMA descriptors of this layer: X, Qb, Tb, unused
+  long long m_pad;       // row pitch of Tb in elements (m rounded up to 8)
   int NB, NP;
 };
 

@@ -273,6 +273,12 @@ __global__ void __launch_bounds__(128) apply_kernel(const DevLayer* __restrict__
       L.Qb[(long long)(L.NP + k) * L.d_in + d] = lo;
     }
   }
+  if (L.Qb) {   // padding rows of the operand panel stay zero
+    for (int k = r; k < L.NP; ++k) {
+      L.Qb[(long long)k * L.d_in + d] = __float2bfloat16_rn(0.f);
+      L.Qb[(long long)(L.NP + k) * L.d_in + d] = __float2bfloat16_rn(0.f);
+    }
+  }
 }
 
 cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s) {

@@ -1,15 +1,522 @@
-// Tensor-core path of Algorithm 1's products with X (placeholder until the tcgen05 kernels land:
-// no layer is eligible, so the CUDA-core path runs).
+// Tensor-core path of Algorithm 1's two products with X on sm_100a: TMA-fed shared-memory
+// tiles, tcgen05.mma with fp32 accumulators in TMEM, one elected thread issuing.
+//
+//   x_q :  T  = H^T Q = X Q        M = 128 tokens, N = NB, K = d_in   (A = X tile, K-major)
+//   xt_t:  Y  = H T   = X^T T      M = 128 columns of X, N = NB, K = tokens
+//                                  (A = the same kind of X tile read as an MN-major operand)
+//
+// X is bf16 and exact; Q and T are fp32 quantities, so each is split as hi + lo in bf16 and
+// the two parts sit side by side as extra N columns (N = NB = 2*NP, NP = r rounded up to 8):
+// the products are exact, the accumulation is fp32, and the column groups are summed in the
+// epilogue.  The kernels are HBM-bound (about r flop per byte of X), so the doubled N is free.
+//
+// Operand panels: Qb [NB][d_in] bf16 (written by the panel-QR apply kernel) and
+// Tt [NB][m_pad] bf16 (T transposed; written by x_q's epilogue or by the Omega fill), both
+// K-major B operands.  Every wait on an mbarrier is bounded; a wait that runs out sets the
+// status word and the CTA leaves through the common exit (TMEM freed).
+#include <cuda.h>
+
+#include <cstring>
+
 #include "agzo_tc.cuh"
 
 namespace agzo {
 
-cudaError_t tc_init(TcState* st, int device) { st->device = device; st->available = false; return cudaSuccess; }
-bool tc_eligible(const agzo_layer&) { return false; }
-size_t tc_layer_scratch(const agzo_layer&) { return 0; }
-void tc_carve(const agzo_layer&, DevLayer* D, char*) { D->Qb = nullptr; D->Tb = nullptr; D->NB = 0; D->NP = 0; }
-cudaError_t tc_fill_omega(const TcState&, const ExtractWave&, const DevLayer*, uint64_t, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t tc_xt_t(const TcState&, const ExtractWave&, const DevLayer*, DevStatus*, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t tc_x_q(const TcState&, const ExtractWave&, const DevLayer*, DevStatus*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kTcThreads = 192;        // warp 0: TMA producer, warp 1: MMA issuer, warps 2..5: epilogue
+constexpr int kBoxK = 64;              // elements per 128-byte swizzle row
+constexpr int kTileBytes = 64 * kBoxK * 2;   // one [64 rows][64 elems] bf16 box = 8 KiB
+constexpr unsigned long long kWaitCapNs = 2000000000ull;   // two seconds
+constexpr size_t kMinSmem = 80 * 1024;  // keeps at most 2 CTAs per SM: 2 * 128 TMEM columns fit
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when two seconds have passed without the phase completing.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > kWaitCapNs) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const void* tmap, int c0, int c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tmap_acquire(const void* tmap) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tmap) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+               "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                         uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+  uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  v[0] = __uint_as_float(r0); v[1] = __uint_as_float(r1); v[2] = __uint_as_float(r2); v[3] = __uint_as_float(r3);
+  v[4] = __uint_as_float(r4); v[5] = __uint_as_float(r5); v[6] = __uint_as_float(r6); v[7] = __uint_as_float(r7);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major operands: 8-row groups are
+// 1024 bytes apart (stride offset), the leading offset is unused.  MN-major operands: rows of
+// the tile are K indices holding 64 contiguous MN elements; `lbo` is the distance between
+// 64-element MN blocks and `sbo` the distance between 8-row K groups.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;          // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;          // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B.
+__device__ __forceinline__ uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+  uint32_t d = 0;
+  d |= 1u << 4;                    // D format: f32
+  d |= 1u << 7;                    // A format: bf16
+  d |= 1u << 10;                   // B format: bf16
+  d |= (uint32_t)(a_mn_major & 1) << 15;
+  d |= (uint32_t)(b_mn_major & 1) << 16;
+  d |= (uint32_t)(N >> 3) << 17;
+  d |= (uint32_t)(M >> 4) << 24;
+  return d;
+}
+
+struct TcShared {
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t accum;
+  uint32_t tmem_base;
+  int failed;
+};
+
+__device__ __forceinline__ uint32_t pow2_cols(int n) {
+  uint32_t c = 32;
+  while ((int)c < n) c <<= 1;
+  return c;
+}
+
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16* hi, __nv_bfloat16* lo) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  *hi = h;
+  *lo = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+
+// ---------------------------------------------------------------- T = X Q  (Tt = T^T as bf16 hi/lo)
+// One CTA per 128-token tile of one layer.  grid = (max token tiles, layers in the wave).
+__global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __restrict__ layers, int l0,
+                                                            DevStatus* status, int stages) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const int t0 = blockIdx.x * 128;
+  if (t0 >= L.m) return;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ TcShared sh;
+  const int NB = L.NB, NP = L.NP;
+  const int a_bytes = 2 * kTileBytes;                 // [128 tokens][64 d]
+  const int b_bytes = NB * kBoxK * 2;                 // [NB][64 d]
+  const int stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023);
+  const int nk = (L.d_in + kBoxK - 1) / kBoxK;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint8_t* maps = reinterpret_cast<const uint8_t*>(L.tmaps);
+  const void* map_x = maps;            // X  [m][d_in], box 64 x 64
+  const void* map_q = maps + 128;      // Qb [NB][d_in], box 64 x NB
+  const uint32_t ncols = pow2_cols(NB);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    mbar_init(&sh.accum, 1);
+    sh.failed = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(&sh.tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tmap_acquire(map_x);
+      tmap_acquire(map_q);
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % stages;
+        if (k >= stages && !mbar_wait(&sh.empty[s], ((k / stages) - 1) & 1)) { sh.failed = 1; break; }
+        uint8_t* a = tiles + (size_t)s * stage_bytes;
+        mbar_expect_tx(&sh.full[s], a_bytes + b_bytes);
+        tma_load_2d(a, map_x, k * kBoxK, t0, &sh.full[s]);
+        tma_load_2d(a + kTileBytes, map_x, k * kBoxK, t0 + 64, &sh.full[s]);
+        tma_load_2d(a + a_bytes, map_q, k * kBoxK, 0, &sh.full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(128, NB, 0, 0);
+      bool ok = true;
+      for (int k = 0; k < nk && ok; ++k) {
+        const int s = k % stages;
+        if (!mbar_wait(&sh.full[s], (k / stages) & 1)) { sh.failed = 1; ok = false; break; }
+        tc_fence_after();
+        const uint32_t a = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint32_t b = a + a_bytes;
+#pragma unroll
+        for (int kk = 0; kk < kBoxK / 16; ++kk) {
+          const uint64_t ad = smem_desc(a + kk * 32, 0, 1024);
+          const uint64_t bd = smem_desc(b + kk * 32, 0, 1024);
+          mma_bf16(tmem, ad, bd, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+        }
+        mma_commit(&sh.empty[s]);      // the stage is free once these MMAs have read it
+      }
+      mma_commit(&sh.accum);           // arrives when every MMA issued so far is done
+    }
+  } else {
+    // epilogue: TMEM lane i of this warp's quarter = token t0 + 32*q + lane
+    const int q = warp & 3;
+    const bool ok = mbar_wait(&sh.accum, 0);
+    tc_fence_after();
+    if (!ok) sh.failed = 1;
+    const int t = t0 + q * 32 + lane;
+    __nv_bfloat16* Tt = L.Tb;
+    const long long mp = L.m_pad;
+    if (ok) {
+      for (int k0 = 0; k0 < NP; k0 += 8) {
+        float hi[8], lo[8];
+        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)k0, hi);
+        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(NP + k0), lo);
+        if (t < L.m) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            __nv_bfloat16 h, l;
+            split_bf16(hi[j] + lo[j], &h, &l);
+            Tt[(long long)(k0 + j) * mp + t] = h;
+            Tt[(long long)(NP + k0 + j) * mp + t] = l;
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (sh.failed && threadIdx.x == 0) { atomicExch(&status->timeout, 1); atomicExch(&status->where, 1); }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, ncols); }
+}
+
+// ---------------------------------------------------------------- Ypart[s] = X_s^T T_s
+// One CTA per (128 columns of X, token slab) of one layer.  grid = (column chunks, slabs, layers).
+__global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __restrict__ layers, int l0,
+                                                             DevStatus* status, int stages) {
+  const DevLayer& L = layers[l0 + blockIdx.z];
+  const int d0 = blockIdx.x * 128;
+  const int slab = blockIdx.y;
+  if (d0 >= L.d_in || slab >= L.slabs) return;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ TcShared sh;
+  const int NB = L.NB, NP = L.NP;
+  const int a_bytes = 2 * kTileBytes;                 // two [64 tokens][64 d] boxes: d0.., d0+64..
+  const int b_bytes = NB * kBoxK * 2;                 // [NB][64 tokens]
+  const int stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023);
+  const int t_begin = slab * L.slab_rows;
+  const int t_end = min(L.m, t_begin + L.slab_rows);
+  const int nk = (t_end - t_begin + kBoxK - 1) / kBoxK;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint8_t* maps = reinterpret_cast<const uint8_t*>(L.tmaps);
+  const void* map_x = maps;            // X  [m][d_in], box 64 x 64
+  const void* map_t = maps + 256;      // Tt [NB][m],   box 64 x NB
+  const uint32_t ncols = pow2_cols(NB);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    mbar_init(&sh.accum, 1);
+    sh.failed = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(&sh.tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tmap_acquire(map_x);
+      tmap_acquire(map_t);
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % stages;
+        if (k >= stages && !mbar_wait(&sh.empty[s], ((k / stages) - 1) & 1)) { sh.failed = 1; break; }
+        uint8_t* a = tiles + (size_t)s * stage_bytes;
+        const int tk = t_begin + k * kBoxK;
+        mbar_expect_tx(&sh.full[s], a_bytes + b_bytes);
+        tma_load_2d(a, map_x, d0, tk, &sh.full[s]);
+        tma_load_2d(a + kTileBytes, map_x, d0 + 64, tk, &sh.full[s]);
+        tma_load_2d(a + a_bytes, map_t, tk, 0, &sh.full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(128, NB, 1, 0);     // A is MN-major: the X tile as X^T
+      bool ok = true;
+      for (int k = 0; k < nk && ok; ++k) {
+        const int s = k % stages;
+        if (!mbar_wait(&sh.full[s], (k / stages) & 1)) { sh.failed = 1; ok = false; break; }
+        tc_fence_after();
+        const uint32_t a = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint32_t b = a + a_bytes;
+#pragma unroll
+        for (int kk = 0; kk < kBoxK / 16; ++kk) {
+          // 16 tokens = two 8-row swizzle atoms = 2048 bytes further down the X boxes
+          const uint64_t ad = smem_desc(a + kk * 2048, kTileBytes, 1024);
+          const uint64_t bd = smem_desc(b + kk * 32, 0, 1024);
+          mma_bf16(tmem, ad, bd, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+        }
+        mma_commit(&sh.empty[s]);
+      }
+      mma_commit(&sh.accum);
+    }
+  } else {
+    const int q = warp & 3;
+    const bool ok = mbar_wait(&sh.accum, 0);
+    tc_fence_after();
+    if (!ok) sh.failed = 1;
+    const int d = d0 + q * 32 + lane;
+    const int r = L.r;
+    if (ok) {
+      float* out = L.Ypart + (long long)slab * r * L.d_in + d;
+      for (int k0 = 0; k0 < NP; k0 += 8) {
+        float hi[8], lo[8];
+        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)k0, hi);
+        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(NP + k0), lo);
+        if (d < L.d_in) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (k0 + j < r) out[(long long)(k0 + j) * L.d_in] = hi[j] + lo[j];
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (sh.failed && threadIdx.x == 0) { atomicExch(&status->timeout, 1); atomicExch(&status->where, 2); }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, ncols); }
+}
+
+// ---------------------------------------------------------------- Omega -> Tt (hi/lo), pads zero
+__global__ void tc_fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const long long n = (long long)L.m * L.r;
+  const long long nb = (n + 3) >> 2;
+  const long long mp = L.m_pad;
+  const int r = L.r, NP = L.NP;
+  for (long long b = blockIdx.x * (long long)blockDim.x + threadIdx.x; b < nb;
+       b += (long long)gridDim.x * blockDim.x) {
+    const float4 g = gaussian_block((uint64_t)b, L.layer_id, kTagOmega, seed);
+    const float gv[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+    for (int lane = 0; lane < 4; ++lane) {
+      const long long e = 4 * b + lane;
+      if (e < n) {
+        const long long t = e / r;
+        const int k = (int)(e - t * r);
+        __nv_bfloat16 h, l;
+        split_bf16(gv[lane], &h, &l);
+        L.Tb[(long long)k * mp + t] = h;
+        L.Tb[(long long)(NP + k) * mp + t] = l;
+      }
+    }
+  }
+  const int pad = NP - r;
+  if (pad > 0) {
+    const long long np = (long long)pad * L.m;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < np;
+         i += (long long)gridDim.x * blockDim.x) {
+      const int k = r + (int)(i / L.m);
+      const long long t = i % L.m;
+      L.Tb[(long long)k * mp + t] = __float2bfloat16_rn(0.f);
+      L.Tb[(long long)(NP + k) * mp + t] = __float2bfloat16_rn(0.f);
+    }
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool encode_2d(void* fn, void* out, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+               uint32_t box_inner, uint32_t box_outer) {
+  CUtensorMap m;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {box_inner, box_outer};
+  const cuuint32_t es[2] = {1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                                                   dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  std::memcpy(out, &m, sizeof(m));
+  return true;
+}
+
+int np_of(int r) { return (r + 7) & ~7; }
+long long mpad_of(int m) { return ((long long)m + 7) & ~7ll; }
+size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+int stages_for(int NB) {
+  const int stage = 2 * kTileBytes + ((NB * kBoxK * 2 + 1023) & ~1023);
+  int s = (int)((96 * 1024) / stage);
+  if (s > 8) s = 8;
+  if (s < 2) s = 2;
+  return s;
+}
+size_t smem_for(int NB, int stages) {
+  const size_t stage = 2 * kTileBytes + ((NB * kBoxK * 2 + 1023) & ~1023);
+  size_t b = stage * stages + 1024;
+  return b < kMinSmem ? kMinSmem : b;
+}
+
+}  // namespace
+
+cudaError_t tc_init(TcState* st, int device) {
+  st->device = device;
+  st->available = false;
+  st->encode_fn = nullptr;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    return cudaSuccess;   // the CUDA-core path still works
+  }
+  int major = 0;
+  cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+  st->encode_fn = fn;
+  st->available = major == 10;
+  if (st->available) {
+    e = cudaFuncSetAttribute(tc_x_q_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(tc_xt_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) { cudaGetLastError(); st->available = false; }
+  }
+  return cudaSuccess;
+}
+
+bool tc_eligible(const agzo_layer& a) {
+  return a.X && a.x_dtype == AGZO_BF16 && (reinterpret_cast<uintptr_t>(a.X) & 15u) == 0 && a.ldx % 8 == 0 &&
+         a.d_in % 8 == 0 && a.d_in >= 128 && a.m >= 256 && a.r >= 1 && a.r <= AGZO_MAX_RANK;
+}
+
+size_t tc_layer_scratch(const agzo_layer& a) {
+  const size_t NB = 2 * (size_t)np_of(a.r);
+  return up256(NB * (size_t)a.d_in * 2) + up256(NB * (size_t)mpad_of(a.m) * 2);
+}
+
+void tc_carve(const agzo_layer& a, DevLayer* D, char* p) {
+  D->NP = np_of(a.r);
+  D->NB = 2 * D->NP;
+  D->m_pad = mpad_of(a.m);
+  D->Qb = reinterpret_cast<__nv_bfloat16*>(p);
+  p += up256((size_t)D->NB * a.d_in * 2);
+  D->Tb = reinterpret_cast<__nv_bfloat16*>(p);
+}
+
+bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps) {
+  if (!st.encode_fn) return false;
+  uint8_t* out = static_cast<uint8_t*>(host_maps);
+  // X [m][ldx]: inner = d_in, outer = m; one box = 64 columns x 64 tokens
+  if (!encode_2d(st.encode_fn, out, D.X, (uint64_t)D.d_in, (uint64_t)D.m, (uint64_t)D.ldx * 2, 64, 64)) return false;
+  // Qb [NB][d_in]: box = 64 columns x NB rows
+  if (!encode_2d(st.encode_fn, out + 128, D.Qb, (uint64_t)D.d_in, (uint64_t)D.NB, (uint64_t)D.d_in * 2, 64,
+                 (uint32_t)D.NB))
+    return false;
+  // Tt [NB][m_pad]: inner extent is the true m so that the padding is read as zero
+  if (!encode_2d(st.encode_fn, out + 256, D.Tb, (uint64_t)D.m, (uint64_t)D.NB, (uint64_t)D.m_pad * 2, 64,
+                 (uint32_t)D.NB))
+    return false;
+  return true;
+}
+
+cudaError_t tc_fill_omega(const TcState&, const ExtractWave& w, const DevLayer*, uint64_t seed, cudaStream_t s) {
+  const long long nb = ((long long)w.max_m * w.max_r + 3) >> 2;
+  int gx = (int)((nb + 255) / 256);
+  if (gx > 1024) gx = 1024;
+  if (gx < 1) gx = 1;
+  tc_fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed);
+  return cudaGetLastError();
+}
+
+cudaError_t tc_xt_t(const TcState&, const ExtractWave& w, const DevLayer* h_dev, DevStatus* d_status,
+                    cudaStream_t s) {
+  int max_nb = 0;
+  for (int i = w.l0; i < w.l1; ++i) max_nb = h_dev[i].NB > max_nb ? h_dev[i].NB : max_nb;
+  const int stages = stages_for(max_nb);
+  dim3 grid((w.max_din + 127) / 128, w.max_slabs, w.l1 - w.l0);
+  tc_xt_t_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages);
+  return cudaGetLastError();
+}
+
+cudaError_t tc_x_q(const TcState&, const ExtractWave& w, const DevLayer* h_dev, DevStatus* d_status,
+                   cudaStream_t s) {
+  int max_nb = 0;
+  for (int i = w.l0; i < w.l1; ++i) max_nb = h_dev[i].NB > max_nb ? h_dev[i].NB : max_nb;
+  const int stages = stages_for(max_nb);
+  dim3 grid((w.max_m + 127) / 128, w.l1 - w.l0);
+  tc_x_q_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages);
+  return cudaGetLastError();
+}
 
 }  // namespace agzo

@@ -18,6 +18,9 @@ size_t tc_layer_scratch(const agzo_layer& a);
 // assigns Qb / Tb / NB / NP of D from scratch starting at p (after the common slices)
 void tc_carve(const agzo_layer& a, DevLayer* D, char* p);
 
+// writes the layer's TMA descriptors (512 bytes) into host memory; false when encoding fails
+bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps);
+
 cudaError_t tc_fill_omega(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,
                           uint64_t seed, cudaStream_t s);
 cudaError_t tc_xt_t(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,

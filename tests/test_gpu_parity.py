@@ -203,6 +203,16 @@ EXTRACT_CASES = [
     (640, 256, 24, 1, 32, True, 1),
     (300, 128, 64, 1, 0, False, 1),
     (400, 96, 5, 0, 0, False, 1),        # K = 0: just qr(H Omega)
+    # the tensor-core kernels (bf16 X, 16-byte aligned rows)
+    (2048, 1024, 8, 0, 32, True, 2),     # K = 0: Omega fill + X^T T + panel QR
+    (2048, 1024, 8, 1, 32, True, 2),     # K = 1 adds X Q
+    (2048, 1024, 8, 3, 32, True, 2),
+    (700, 520, 8, 3, 16, True, 2),       # ragged tiles, padded pitch
+    (1000, 384, 1, 3, 8, True, 2),
+    (333, 200, 16, 2, 32, True, 2),
+    (640, 256, 24, 1, 32, True, 2),
+    (512, 256, 64, 1, 0, True, 2),
+    (4096, 3072, 4, 3, 32, True, 2),     # several column chunks and slabs
 ]
 
 
