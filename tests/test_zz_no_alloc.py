@@ -39,10 +39,12 @@ def test_static_scratch_variant_matches_the_regular_entry_point_twice_in_a_row()
         Vbuf = torch.full((r + 2, d_in + 4), 7.0, device=DEV)
         V = Vbuf[1:1 + r, :d_in]
         flag = torch.full((1,), -1, dtype=torch.int32, device=DEV)
-        before = torch.cuda.memory_allocated()
+        # cumulative count of allocations made through torch: frees by the garbage collector in
+        # the meantime cannot move it, a new allocation would
+        before = torch.cuda.memory_stats()["allocation.all.allocated"]
         B.agzo_extract_subspace_static(Xd, V, r, K, seed, layer_id, d_rank_deficient=flag)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
         got = to_host(V)
         assert int(flag) == 0
         assert np.abs(got.astype(np.float64) @ got.T - np.eye(r)).max() <= 1e-5
