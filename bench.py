@@ -180,10 +180,16 @@ def main():
     ap.add_argument("--rank", type=int, default=16)
     ap.add_argument("--extract-path", type=int, default=0)
     ap.add_argument("--wave-mb", type=int, default=-1)
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="keep only the first N transformer blocks of the layer set (profiling-sized runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     cfg = WL.LAYER_SETS[args.workload]
+    if args.blocks > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, n_blocks=min(args.blocks, cfg.n_blocks),
+                                  name=f"{cfg.name}[first {min(args.blocks, cfg.n_blocks)} blocks]")
     r = args.rank
     if args.impl == "reference":
         return run_reference(args, cfg, r)

@@ -16,7 +16,7 @@ constexpr uint32_t kMagic = 0xA620B200u;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;          // DevStatus + scalar slots
 constexpr size_t kCoefOffset = 64;            // float coefficient slot inside the header
-constexpr int64_t kDefaultWaveBytes = 48ll << 20;
+constexpr int64_t kDefaultWaveBytes = 4ll << 30;
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
@@ -132,13 +132,12 @@ agzo_status validate(const agzo_layer* L, int n, int need) {
 bool has_x(const agzo_layer& a) { return a.X != nullptr && a.m >= 1; }
 
 // Token slabs of the X^T T product.  CUDA-core kernels: 32 slabs at most.  Tensor-core
-// kernels: enough (column chunk, slab) CTAs to fill the GPU twice, slabs a multiple of 64 tokens.
+// kernels: slabs of 2048 tokens (32 pipeline steps per CTA) when the layer has that many; a
+// wave holds many layers, so the grid is filled by the layers, not by thin slabs.
 void slab_shape(const agzo_layer& a, bool tc, int* slabs, int* slab_rows) {
   int rows;
   if (tc) {
-    const int chunks = (a.d_in + 127) / 128;
-    const int want = (2 * 148 + chunks - 1) / chunks;
-    rows = (a.m + want - 1) / want;
+    rows = a.m >= 8192 ? 2048 : (a.m + 3) / 4;
     rows = (rows + 63) / 64 * 64;
   } else {
     rows = (a.m + 31) / 32;
@@ -228,8 +227,10 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
     size_t used = 0;
     int64_t xbytes = 0;
     int j = i;
+    const bool wave_tc = extract_path != 1 && tc_available && tc_eligible(L[i]);
     while (j < n && has_x(L[j])) {
       const bool tc = extract_path != 1 && tc_available && tc_eligible(L[j]);
+      if (tc != wave_tc) break;      // a wave runs on one kind of kernel
       const size_t need = layer_scratch(L[j], tc);
       const int64_t xb = (int64_t)L[j].m * L[j].d_in * (L[j].x_dtype == AGZO_BF16 ? 2 : 4);
       if (j > i && (used + need > scratch_cap || xbytes + xb > wave_bytes)) break;
@@ -368,10 +369,15 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   if (!h_bytes) return AGZO_ERR_INVALID_ARG;
   agzo_status st = validate(h_layers, n, 0);
   if (st != AGZO_OK) return st;
+  // large enough for either kind of extraction kernel (the "extract_path" option may pick
+  // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
-  size_t scratch = 0;
+  size_t scratch = 0, scratch_cc = 0;
   st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 0, true, &plan, &scratch);
   if (st != AGZO_OK) return st;
+  st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 1, false, &plan, &scratch_cc);
+  if (st != AGZO_OK) return st;
+  if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
   return AGZO_OK;
 }
