@@ -120,6 +120,10 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
 
 /* Options: "extract_path" 0 = automatic, 1 = CUDA-core fp32 kernels only, 2 = require the
  * tensor-core kernels (UNSUPPORTED at call time if a layer cannot use them);
+ * "rmw_path" selects the kernel of the in-place passes: 0 = automatic (bf16 weights with
+ * 16-byte aligned rows and r >= "rmw_tc_min_rank", default 8, take the tensor-core kernel,
+ * everything else the CUDA-core kernels), 1 = CUDA-core kernels only, 2 = tensor-core kernel
+ * for every layer that allows it;
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
  * "time_kernel_class" = one agzo_kernel_class whose launches get a CUDA event pair on the
  * caller's stream (0 = none), read back by agzo_read_counters.                           */
@@ -133,7 +137,8 @@ typedef enum agzo_kernel_class {
   AGZO_KC_PANEL_QR = 4,   /* the three kernels of qr(Y) as one unit                        */
   AGZO_KC_TC_XT_T = 5,    /* Y = X^T T, tensor-core kernel                                 */
   AGZO_KC_TC_X_Q = 6,     /* T = X Q, tensor-core kernel                                   */
-  AGZO_KC_OMEGA = 7       /* Gaussian test matrix fill                                     */
+  AGZO_KC_OMEGA = 7,      /* Gaussian test matrix fill                                     */
+  AGZO_KC_RMW_TC = 8      /* the in-place low-rank pass, tensor-core kernel                */
 } agzo_kernel_class;
 
 /* Measurement aid.  Waits for the timed launches recorded since the last read, then returns

@@ -29,6 +29,18 @@ struct Plan {
   int fast_mode_mask = 0;          // storage modes present among layers on the vector path
   bool any_slow = false;           // some layer needs the scalar kernel
   bool has_extract = false;
+  // tensor-core in-place pass: work items per layer (prefix, n + 1), zero-length for other layers
+  std::vector<int> item_start;
+  int total_items = 0;
+  int max_rp = 0;
+};
+
+struct PlanOpts {
+  int64_t wave_bytes;
+  int extract_path;      // 0 auto, 1 CUDA-core only, 2 tensor-core required
+  int rmw_path;          // 0 auto, 1 CUDA-core only, 2 tensor cores wherever a layer allows it
+  int rmw_tc_min_rank;   // auto: layers with r >= this use the tensor-core pass
+  bool tc_available;
 };
 
 }  // namespace
@@ -41,6 +53,8 @@ struct agzo_ctx {
   size_t ws_bytes;
   int last_cuda;
   int extract_path;        // 0 auto, 1 CUDA-core only, 2 tensor-core required
+  int rmw_path;            // 0 auto, 1 CUDA-core only, 2 tensor cores wherever possible
+  int rmw_tc_min_rank;
   int64_t wave_bytes;
   // descriptors last uploaded
   std::vector<agzo_layer> cached;
@@ -166,17 +180,19 @@ size_t layer_scratch(const agzo_layer& a, bool tc) {
 }
 
 constexpr size_t kMapBytes = 512;   // four TMA descriptors per layer
+// device tables after the header: layer records | tile prefix and item prefix (n + 1 ints each) | TMA descriptors
+size_t prefix_bytes(int n) { return align_up((size_t)2 * (n + 1) * sizeof(int)); }
 size_t table_bytes(int n) {
-  return align_up((size_t)n * sizeof(DevLayer)) + align_up((size_t)(n + 1) * sizeof(int)) +
-         align_up((size_t)n * kMapBytes);
+  return align_up((size_t)n * sizeof(DevLayer)) + prefix_bytes(n) + align_up((size_t)n * kMapBytes);
 }
-size_t maps_offset(int n) {
-  return kHeaderBytes + align_up((size_t)n * sizeof(DevLayer)) + align_up((size_t)(n + 1) * sizeof(int));
-}
+size_t maps_offset(int n) { return kHeaderBytes + align_up((size_t)n * sizeof(DevLayer)) + prefix_bytes(n); }
 
 // Builds the device records.  ws == nullptr: only sizes are computed (scratch_needed).
-agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, int64_t wave_bytes,
-                       int extract_path, bool tc_available, Plan* plan, size_t* scratch_needed) {
+agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, const PlanOpts& opts,
+                       Plan* plan, size_t* scratch_needed) {
+  const int64_t wave_bytes = opts.wave_bytes;
+  const int extract_path = opts.extract_path;
+  const bool tc_available = opts.tc_available;
   plan->dev.assign(n, DevLayer{});
   plan->tile_start.assign(n + 1, 0);
   plan->wave_end.clear();
@@ -184,11 +200,15 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
   plan->fast_mode_mask = 0;
   plan->any_slow = false;
   plan->has_extract = false;
+  plan->item_start.assign(n + 1, 0);
+  plan->total_items = 0;
+  plan->max_rp = 0;
   const size_t base = kHeaderBytes + table_bytes(n);
   const size_t scratch_cap = ws ? (ws_bytes > base ? ws_bytes - base : 0) : (size_t)-1;
   size_t max_wave_scratch = 0;
 
   int tiles = 0;
+  long long items = 0;
   for (int i = 0; i < n; ++i) {
     const agzo_layer& a = L[i];
     DevLayer& D = plan->dev[i];
@@ -203,12 +223,23 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
                aligned16(a.V) && a.ldv % 4 == 0;
     if (a.W16) vec = vec && aligned16(a.W16) && (a.ldw16 * 2) % 16 == 0;
     D.vec_ok = vec ? 1 : 0;
-    if (a.W) {
+    // bf16 weights of sufficient rank go through the tensor-core pass and get no CUDA-core tiles
+    const bool tc_rmw = tc_available && opts.rmw_path != 1 && rmw_tc_eligible(a) &&
+                        (opts.rmw_path == 2 || a.r >= opts.rmw_tc_min_rank);
+    plan->item_start[i] = (int)items;
+    if (tc_rmw) {
+      rmw_tc_shape(a, &D);
+      D.rtc_item0 = (int)items;
+      items += (long long)D.rtc_panels * D.rtc_chunks;
+      if (items > 0x7fffffff) return AGZO_ERR_INVALID_ARG;
+      if (D.rtc_rp > plan->max_rp) plan->max_rp = D.rtc_rp;
+      if (ws) D.wmap = ws + maps_offset(n) + (size_t)i * kMapBytes + 384;
+    } else if (a.W) {
       if (vec) plan->fast_mode_mask |= 1 << D.rmw_mode; else plan->any_slow = true;
     }
     D.tile0 = tiles;
     D.tiles_c = (a.d_in + 511) / 512;
-    D.tiles_r = a.W ? (a.d_out + 255) / 256 : 0;
+    D.tiles_r = (a.W && !tc_rmw) ? (a.d_out + 255) / 256 : 0;
     plan->tile_start[i] = tiles;
     const long long nt = (long long)D.tiles_c * D.tiles_r;
     if (tiles + nt > 0x7fffffff) return AGZO_ERR_INVALID_ARG;
@@ -217,6 +248,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, in
   }
   plan->tile_start[n] = tiles;
   plan->total_tiles = tiles;
+  plan->item_start[n] = (int)items;
+  plan->total_items = (int)items;
 
   // extraction waves: consecutive layers whose activations fit the wave budget and whose
   // scratch fits the workspace
@@ -276,6 +309,7 @@ DevLayer* dev_layers(agzo_ctx* c) { return reinterpret_cast<DevLayer*>(c->ws + k
 int* dev_tiles(agzo_ctx* c, int n) {
   return reinterpret_cast<int*>(c->ws + kHeaderBytes + align_up((size_t)n * sizeof(DevLayer)));
 }
+int* dev_items(agzo_ctx* c, int n) { return dev_tiles(c, n) + (n + 1); }
 DevStatus* dev_status(agzo_ctx* c) { return reinterpret_cast<DevStatus*>(c->ws); }
 float* dev_coef(agzo_ctx* c) { return reinterpret_cast<float*>(c->ws + kCoefOffset); }
 
@@ -284,11 +318,11 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (same_layers(c, L, n)) return AGZO_OK;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
-  agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, c->wave_bytes, c->extract_path,
-                              c->tc.available, &plan, nullptr);
+  const PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->tc.available};
+  agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st != AGZO_OK) return st;
   const size_t lb = align_up((size_t)n * sizeof(DevLayer));
-  const size_t tb = align_up((size_t)(n + 1) * sizeof(int)) + (size_t)n * kMapBytes;
+  const size_t tb = prefix_bytes(n) + (size_t)n * kMapBytes;
   if (c->stage_pending) {
     CU(c, cudaEventSynchronize(c->stage_ev));
     c->stage_pending = false;
@@ -305,10 +339,13 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
     char* hs = static_cast<char*>(c->h_stage);
     std::memset(hs + lb, 0, tb);
     std::memcpy(hs + lb, plan.tile_start.data(), (size_t)(n + 1) * sizeof(int));
-    char* hmaps = hs + lb + align_up((size_t)(n + 1) * sizeof(int));
+    std::memcpy(hs + lb + (size_t)(n + 1) * sizeof(int), plan.item_start.data(), (size_t)(n + 1) * sizeof(int));
+    char* hmaps = hs + lb + prefix_bytes(n);
     for (int i = 0; i < n; ++i) {
-      if (!plan.dev[i].Qb) continue;
-      if (!tc_encode_maps(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes)) return AGZO_ERR_UNSUPPORTED;
+      if (plan.dev[i].Qb && !tc_encode_maps(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes))
+        return AGZO_ERR_UNSUPPORTED;
+      if (plan.dev[i].wmap && !rmw_tc_encode_map(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes + 384))
+        return AGZO_ERR_UNSUPPORTED;
     }
     CU(c, cudaMemcpyAsync(c->ws + kHeaderBytes, c->h_stage, lb + tb, cudaMemcpyHostToDevice, s));
     CU(c, cudaEventRecord(c->stage_ev, s));
@@ -336,10 +373,17 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   if (n == 0) return AGZO_OK;
   st = prepare(c, L, n, s);
   if (st != AGZO_OK) return st;
-  Timed t(c, AGZO_KC_RMW, s);
-  CU(c, launch_rmw(dev_layers(c), dev_tiles(c, n), n, c->plan.total_tiles, c->plan.max_r,
-                   c->plan.fast_mode_mask, c->plan.any_slow, seed, coef, d_coef, pair_update,
-                   c->sm_count, s));
+  if (c->plan.total_items > 0) {
+    Timed t(c, AGZO_KC_RMW_TC, s);
+    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, seed, coef,
+                        d_coef, dev_status(c), c->sm_count, s));
+  }
+  if (c->plan.total_tiles > 0) {
+    Timed t(c, AGZO_KC_RMW, s);
+    CU(c, launch_rmw(dev_layers(c), dev_tiles(c, n), n, c->plan.total_tiles, c->plan.max_r,
+                     c->plan.fast_mode_mask, c->plan.any_slow, seed, coef, d_coef, pair_update,
+                     c->sm_count, s));
+  }
   return AGZO_OK;
 }
 
@@ -373,9 +417,9 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 0, true, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, true}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, kDefaultWaveBytes, 1, false, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, false}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -399,6 +443,8 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->ws_bytes = workspace_bytes;
   c->last_cuda = 0;
   c->extract_path = 0;
+  c->rmw_path = 0;
+  c->rmw_tc_min_rank = 8;
   c->wave_bytes = kDefaultWaveBytes;
   c->cached_valid = false;
   c->h_stage = nullptr;
@@ -440,11 +486,17 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
   if (std::strcmp(name, "extract_path") == 0) {
     if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
     ctx->extract_path = (int)value;
+  } else if (std::strcmp(name, "rmw_path") == 0) {
+    if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
+    ctx->rmw_path = (int)value;
+  } else if (std::strcmp(name, "rmw_tc_min_rank") == 0) {
+    if (value < 1 || value > AGZO_MAX_RANK) return AGZO_ERR_INVALID_ARG;
+    ctx->rmw_tc_min_rank = (int)value;
   } else if (std::strcmp(name, "wave_bytes") == 0) {
     if (value < 0) return AGZO_ERR_INVALID_ARG;
     ctx->wave_bytes = value;
   } else if (std::strcmp(name, "time_kernel_class") == 0) {
-    if (value < 0 || value > 7) return AGZO_ERR_INVALID_ARG;
+    if (value < 0 || value > 8) return AGZO_ERR_INVALID_ARG;
     ctx->time_class = (int)value;
     return AGZO_OK;
   } else {

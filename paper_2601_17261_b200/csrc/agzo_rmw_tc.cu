@@ -1,0 +1,416 @@
+// In-place low-rank pass W <- W + c * R A^T (Eq. agzo-perturb, Algorithm 2) for bf16 weights
+// with the rank-r outer product on the tensor cores of sm_100a.
+//
+// The CUDA-core kernel (agzo_rmw.cu) spends r + 1 fp32 FMAs per weight; from r = 16 on that is
+// more arithmetic than the FP32 pipes can do in the time HBM needs to stream the weight once in
+// and once out.  Here the product Delta = R A^T of a 128-row tile is one small tcgen05.mma chain
+// (M = 128, N = the panel's columns, K = 4 * rp), its fp32 result waits in TMEM, and the only
+// per-weight work left for the CUDA cores is  w + c * delta  and the rounding to bf16.
+//
+// Precision: R and A^T are fp32; each is split as hi + lo in bf16 and the four cross products
+// are laid side by side along K (K index = [RhAh | RhAl | RlAh | RlAl]), so the products are
+// exact and summed in fp32; what is dropped is below 2^-17 of each term.
+//
+// Data flow of one CTA (persistent, one per SM):
+//   loader thread      TMA-loads 128 x 64 boxes of W into a ring of shared-memory slots
+//   R warps (4)        regenerate the tile's 128 rows of R from the Philox counter and write the
+//                      split A operand; at the start of an item they also build the B operand
+//                      from the panel's slice of A^T (V)
+//   MMA thread         issues the tcgen05.mma chain into one of two TMEM buffers
+//   epilogue warps (8) read delta from TMEM and W from the slot, write the new bf16 W back
+//                      into the slot
+//   storer thread      TMA-stores the slot to the place it was loaded from
+// Every wait on an mbarrier is bounded; a wait that runs out sets the status word and the CTA
+// leaves through the common exit (copies drained, TMEM freed).
+#include <cuda.h>
+
+#include "agzo_ptx.cuh"
+#include "agzo_tc.cuh"
+
+namespace agzo {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kRows = 128;                 // rows of a tile (MMA M)
+constexpr int kBoxCols = 64;               // columns of one W box = one 128-byte swizzle row
+constexpr int kBoxBytes = kRows * 128;     // 16 KiB
+constexpr int kAtomBytesA = kRows * 128;   // one 64-wide K atom of the A operand
+constexpr int kBBytes = 32 * 1024;         // B operand: panel columns x K, always 32 KiB
+constexpr int kMaxSlots = 12;
+constexpr int kWarpLoader = 0, kWarpMma = 1, kWarpStorer = 2, kWarpEpi0 = 3, kNumEpiWarps = 8,
+              kWarpGen0 = kWarpEpi0 + kNumEpiWarps, kNumGenWarps = 4;
+constexpr int kThreads = (kWarpGen0 + kNumGenWarps) * 32;   // 480
+constexpr uint32_t kTmemCols = 512;        // two delta buffers of up to 256 columns
+
+struct Shared {
+  uint64_t full_w[kMaxSlots];    // TMA load of the slot landed
+  uint64_t epi_done[kMaxSlots];  // epilogue warps wrote the slot back
+  uint64_t empty_w[kMaxSlots];   // TMA store has read the slot
+  uint64_t a_full[2], a_empty[2];
+  uint64_t b_full, b_empty;
+  uint64_t tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int failed;
+};
+
+struct Item {
+  const DevLayer* L;
+  int col0, rb0, rb1, cw, rp, nboxes;
+};
+
+__device__ __forceinline__ int find_layer_of_item(const int* start, int n_layers, int item) {
+  int lo = 0, hi = n_layers - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (__ldg(start + mid) <= item) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ Item decode_item(const DevLayer* layers, const int* item_start, int n_layers, int item) {
+  Item it;
+  const DevLayer* L = layers + find_layer_of_item(item_start, n_layers, item);
+  it.L = L;
+  const int local = item - L->rtc_item0;
+  const int chunk = local / L->rtc_panels, panel = local - chunk * L->rtc_panels;
+  it.cw = L->rtc_cw;
+  it.rp = L->rtc_rp;
+  it.col0 = panel * it.cw;
+  const int nrb = (L->d_out + kRows - 1) / kRows;
+  it.rb0 = chunk * L->rtc_chunk_blocks;
+  it.rb1 = min(nrb, it.rb0 + L->rtc_chunk_blocks);
+  const int cols_left = L->d_in - it.col0;
+  it.nboxes = min(it.cw / kBoxCols, (cols_left + kBoxCols - 1) / kBoxCols);
+  return it;
+}
+
+// byte offset of 16-byte chunk j of row i inside a [rows][128 bytes] block with the 128-byte swizzle
+__device__ __forceinline__ uint32_t swz(int i, int j) {
+  return (uint32_t)((i >> 3) * 1024 + (i & 7) * 128 + ((j ^ (i & 7)) << 4));
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);   // a in the low half
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ float lo_part(float v) { return v - __bfloat162float(__float2bfloat16_rn(v)); }
+
+// Eight fp32 values -> their bf16 hi parts and bf16 lo parts (v ~ hi + lo)
+__device__ __forceinline__ void split8(const float (&v)[8], uint4* hi, uint4* lo) {
+  hi->x = pack2(v[0], v[1]); hi->y = pack2(v[2], v[3]); hi->z = pack2(v[4], v[5]); hi->w = pack2(v[6], v[7]);
+  lo->x = pack2(lo_part(v[0]), lo_part(v[1])); lo->y = pack2(lo_part(v[2]), lo_part(v[3]));
+  lo->z = pack2(lo_part(v[4]), lo_part(v[5])); lo->w = pack2(lo_part(v[6]), lo_part(v[7]));
+}
+
+// Writes group g (8 consecutive rank indices) of one operand row: the hi part goes to K terms
+// t0a and t0b, the lo part to t1a and t1b (term t occupies K indices [t*rp, (t+1)*rp)).
+__device__ __forceinline__ void put_group(uint8_t* base, int atom_bytes, int row, int g, int g8, uint4 hi, uint4 lo,
+                                          int t_hi_a, int t_hi_b, int t_lo_a, int t_lo_b) {
+  const int terms[4] = {t_hi_a, t_hi_b, t_lo_a, t_lo_b};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int cg = terms[q] * g8 + g;              // 16-byte chunk index along K
+    uint8_t* p = base + (cg >> 3) * atom_bytes + swz(row, cg & 7);
+    *reinterpret_cast<uint4*>(p) = q < 2 ? hi : lo;
+  }
+}
+
+__device__ __forceinline__ float pick(const float4& g, int lane) {
+  return lane == 0 ? g.x : lane == 1 ? g.y : lane == 2 ? g.z : g.w;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_start, int n_layers,
+              int total_items, int a_bufs, int a_buf_bytes, int slots, uint64_t seed, float coef_imm,
+              const float* __restrict__ d_coef, DevStatus* status) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = base;                                   // a_bufs x a_buf_bytes
+  uint8_t* sB = sA + (size_t)a_bufs * a_buf_bytes;      // kBBytes
+  uint8_t* sW = sB + kBBytes;                           // slots x kBoxBytes
+  __shared__ Shared sh;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < slots; ++s) {
+      mbar_init(&sh.full_w[s], 1);
+      mbar_init(&sh.epi_done[s], kNumEpiWarps);
+      mbar_init(&sh.empty_w[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sh.a_full[b], kNumGenWarps);
+      mbar_init(&sh.a_empty[b], 1);
+      mbar_init(&sh.tmem_full[b], 1);
+      mbar_init(&sh.tmem_empty[b], kNumEpiWarps);
+    }
+    mbar_init(&sh.b_full, kNumGenWarps);
+    mbar_init(&sh.b_empty, 1);
+    sh.failed = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  if (warp == kWarpMma) tmem_alloc(&sh.tmem_base, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp == kWarpLoader) {
+    if (lane == 0) {
+      int n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+        const Item it = decode_item(layers, item_start, n_layers, item);
+        const void* map = it.L->wmap;
+        tmap_acquire(map);
+        for (int rb = it.rb0; rb < it.rb1 && ok; ++rb) {
+          for (int j = 0; j < it.nboxes; ++j, ++n) {
+            const int s = n % slots, u = n / slots;
+            if (u > 0 && !mbar_wait(&sh.empty_w[s], (u - 1) & 1)) { ok = false; break; }
+            mbar_expect_tx(&sh.full_w[s], kBoxBytes);
+            tma_load_2d(sW + (size_t)s * kBoxBytes, map, it.col0 + j * kBoxCols, rb * kRows, &sh.full_w[s]);
+          }
+        }
+      }
+      if (!ok) sh.failed = 1;
+      if (!ok || sh.failed) {   // leaving early: the copies in flight must land before the CTA goes away
+        for (int k = n > slots ? n - slots : 0; k < n; ++k) mbar_wait(&sh.full_w[k % slots], (k / slots) & 1);
+      }
+    }
+  } else if (warp == kWarpStorer) {
+    if (lane == 0) {
+      int n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+        const Item it = decode_item(layers, item_start, n_layers, item);
+        const void* map = it.L->wmap;
+        tmap_acquire(map);
+        for (int rb = it.rb0; rb < it.rb1 && ok; ++rb) {
+          for (int j = 0; j < it.nboxes; ++j, ++n) {
+            const int s = n % slots, u = n / slots;
+            if (!mbar_wait(&sh.epi_done[s], u & 1)) { ok = false; break; }
+            tma_store_2d(map, it.col0 + j * kBoxCols, rb * kRows, sW + (size_t)s * kBoxBytes);
+            tma_commit_group();
+            if (n > 0) {                      // the previous box's store has read its slot
+              tma_wait_group_read<1>();
+              mbar_arrive(&sh.empty_w[(n - 1) % slots]);
+            }
+          }
+        }
+      }
+      tma_wait_group<0>();                    // every store of this CTA is complete
+      if (!ok) sh.failed = 1;
+    }
+  } else if (warp == kWarpMma) {
+    if (lane == 0) {
+      int t = 0, ic = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++ic) {
+        const Item it = decode_item(layers, item_start, n_layers, item);
+        if (!mbar_wait(&sh.b_full, ic & 1)) { ok = false; break; }
+        const uint32_t idesc = instr_desc(kRows, it.cw, 0, 0);
+        const int ksteps = it.rp / 4;                    // K = 4 * rp, 16 per instruction
+        const uint32_t b_atom = (uint32_t)it.cw * 128u;
+        for (int rb = it.rb0; rb < it.rb1; ++rb, ++t) {
+          const int ab = t % a_bufs, au = t / a_bufs;
+          if (!mbar_wait(&sh.a_full[ab], au & 1)) { ok = false; break; }
+          const int tb = t & 1, tu = t >> 1;
+          if (tu > 0 && !mbar_wait(&sh.tmem_empty[tb], (tu - 1) & 1)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(sA + (size_t)ab * a_buf_bytes);
+          const uint32_t b0 = smem_u32(sB);
+          for (int ks = 0; ks < ksteps; ++ks) {
+            const int ka = ks >> 2, kk = ks & 3;
+            const uint64_t ad = smem_desc(a0 + ka * kAtomBytesA + kk * 32, 0, 1024);
+            const uint64_t bd = smem_desc(b0 + ka * b_atom + kk * 32, 0, 1024);
+            mma_bf16(tmem + (uint32_t)tb * 256u, ad, bd, idesc, ks > 0 ? 1u : 0u);
+          }
+          mma_commit(&sh.a_empty[ab]);
+          mma_commit(&sh.tmem_full[tb]);
+        }
+        mma_commit(&sh.b_empty);
+      }
+      if (!ok) sh.failed = 1;
+    }
+  } else if (warp >= kWarpGen0) {
+    // ------------------------------------------------ operand builders: thread gt = row of the tile
+    const int gt = threadIdx.x - kWarpGen0 * 32;
+    int t = 0, ic = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++ic) {
+      const Item it = decode_item(layers, item_start, n_layers, item);
+      const DevLayer& L = *it.L;
+      const int r = L.r, g8 = it.rp >> 3;
+      // B operand: row n = column col0 + n of the panel, K = [Ah | Al | Ah | Al]
+      if (ic > 0) {
+        ok = mbar_wait(&sh.b_empty, (ic - 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      const int b_atom = it.cw * 128;
+      for (int n = gt; n < it.cw; n += kNumGenWarps * 32) {
+        const int col = it.col0 + n;
+        for (int g = 0; g < g8; ++g) {
+          float v[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int k = 8 * g + u;
+            v[u] = (k < r && col < L.d_in) ? __ldg(L.V + (long long)k * L.ldv + col) : 0.f;
+          }
+          uint4 hi, lo;
+          split8(v, &hi, &lo);
+          put_group(sB, b_atom, n, g, g8, hi, lo, 0, 2, 1, 3);
+        }
+      }
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.b_full);
+      // A operand per tile: row i = R[rb*128 + i][:], K = [Rh | Rh | Rl | Rl]
+      for (int rb = it.rb0; rb < it.rb1; ++rb, ++t) {
+        const int ab = t % a_bufs, au = t / a_bufs;
+        if (au > 0) {
+          ok = mbar_wait(&sh.a_empty[ab], (au - 1) & 1);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
+        uint8_t* a_base = sA + (size_t)ab * a_buf_bytes;
+        const long long row = (long long)rb * kRows + gt;
+        const bool live = row < L.d_out;
+        const long long e0 = row * r;
+        long long cur = -1;
+        float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int g = 0; g < g8; ++g) {
+          float v[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int k = 8 * g + u;
+            float x = 0.f;
+            if (live && k < r) {
+              const long long e = e0 + k;
+              if ((e >> 2) != cur) {
+                cur = e >> 2;
+                g4 = gaussian_block((uint64_t)cur, L.layer_id, kTagG, seed);
+              }
+              x = pick(g4, (int)(e & 3));
+            }
+            v[u] = x;
+          }
+          uint4 hi, lo;
+          split8(v, &hi, &lo);
+          put_group(a_base, kAtomBytesA, gt, g, g8, hi, lo, 0, 1, 2, 3);
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.a_full[ab]);
+      }
+    }
+    if (!ok) sh.failed = 1;
+  } else {
+    // ------------------------------------------------ epilogue: thread = row of the tile, 32 columns of each box
+    const int e = warp - kWarpEpi0;
+    const int q = warp & 3;            // TMEM lanes 32q .. 32q+31 belong to this warp
+    const int h = e >> 2;              // which half of a box's 64 columns
+    const int i = q * 32 + lane;       // row inside the tile
+    const float coef = d_coef ? __ldg(d_coef) : coef_imm;
+    int t = 0, n = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      const Item it = decode_item(layers, item_start, n_layers, item);
+      for (int rb = it.rb0; rb < it.rb1 && ok; ++rb, ++t) {
+        const int tb = t & 1, tu = t >> 1;
+        ok = mbar_wait(&sh.tmem_full[tb], tu & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        for (int j = 0; j < it.nboxes; ++j, ++n) {
+          const int s = n % slots, u = n / slots;
+          ok = mbar_wait(&sh.full_w[s], u & 1);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          uint32_t z[32];
+          tmem_ld32_issue(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * 256 + j * kBoxCols + h * 32), z);
+          uint8_t* slot = sW + (size_t)s * kBoxBytes;
+          uint4 w[4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) w[c] = *reinterpret_cast<const uint4*>(slot + swz(i, h * 4 + c));
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t wi[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
+            uint32_t o[4];
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+              const float w0 = __uint_as_float(wi[p] << 16), w1 = __uint_as_float(wi[p] & 0xFFFF0000u);
+              const float o0 = fmaf(coef, __uint_as_float(z[8 * c + 2 * p]), w0);
+              const float o1 = fmaf(coef, __uint_as_float(z[8 * c + 2 * p + 1]), w1);
+              o[p] = pack2(o0, o1);
+            }
+            *reinterpret_cast<uint4*>(slot + swz(i, h * 4 + c)) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.epi_done[s]);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(&sh.tmem_empty[tb]);
+      }
+    }
+    if (!ok) sh.failed = 1;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (sh.failed && threadIdx.x == 0) { atomicExch(&status->timeout, 1); atomicExch(&status->where, 3); }
+  if (warp == kWarpMma) { tc_fence_after(); tmem_dealloc(tmem, kTmemCols); }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- host side
+bool rmw_tc_eligible(const agzo_layer& a) {
+  return a.W && !a.W16 && a.w_dtype == AGZO_BF16 && (reinterpret_cast<uintptr_t>(a.W) & 15u) == 0 &&
+         (a.ldw * 2) % 16 == 0 && a.d_out >= 1 && a.d_in >= 1 && a.r >= 1 && a.r <= AGZO_MAX_RANK;
+}
+
+void rmw_tc_shape(const agzo_layer& a, DevLayer* D) {
+  const int rp = (a.r + 7) & ~7;
+  const int katoms = (4 * rp + 63) / 64;                 // 1, 2, 3 or 4 K atoms of 64
+  const int cw = katoms == 1 ? 256 : katoms == 2 ? 128 : 64;
+  D->rtc_rp = rp;
+  D->rtc_cw = cw;
+  D->rtc_panels = (a.d_in + cw - 1) / cw;
+  D->rtc_chunk_blocks = 8;
+  const int nrb = (a.d_out + kRows - 1) / kRows;
+  D->rtc_chunks = (nrb + D->rtc_chunk_blocks - 1) / D->rtc_chunk_blocks;
+}
+
+bool rmw_tc_encode_map(const TcState& st, const DevLayer& D, void* host_map) {
+  // W [d_out][ldw] bf16: inner = d_in, outer = d_out; one box = 64 columns x 128 rows
+  return tc_encode_bf16_2d(st, host_map, D.W, (uint64_t)D.d_in, (uint64_t)D.d_out, (uint64_t)D.ldw * 2, kBoxCols,
+                           kRows);
+}
+
+cudaError_t rmw_tc_init() {
+  return cudaFuncSetAttribute(rmw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
+}
+
+cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
+                          int max_rp, uint64_t seed, float coef, const float* d_coef, DevStatus* d_status,
+                          int sm_count, cudaStream_t s) {
+  if (total_items <= 0) return cudaSuccess;
+  const int katoms = (4 * max_rp + 63) / 64;
+  const int a_buf_bytes = katoms * kAtomBytesA;
+  const int a_bufs = katoms >= 3 ? 1 : 2;
+  const int fixed = a_bufs * a_buf_bytes + kBBytes;
+  int slots = (224 * 1024 - fixed) / kBoxBytes;
+  if (slots > kMaxSlots) slots = kMaxSlots;
+  const size_t smem = (size_t)fixed + (size_t)slots * kBoxBytes + 1024;
+  const int grid = total_items < sm_count ? total_items : sm_count;
+  rmw_tc_kernel<<<grid, kThreads, smem, s>>>(d_layers, d_item_start, n_layers, total_items, a_bufs, a_buf_bytes,
+                                             slots, seed, coef, d_coef, d_status);
+  return cudaGetLastError();
+}
+
+}  // namespace agzo

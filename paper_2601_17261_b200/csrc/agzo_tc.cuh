@@ -21,6 +21,19 @@ void tc_carve(const agzo_layer& a, DevLayer* D, char* p);
 // writes the layer's TMA descriptors (512 bytes) into host memory; false when encoding fails
 bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps);
 
+// generic bf16 2-D tiled descriptor with the 128-byte swizzle (128 bytes written to `out`)
+bool tc_encode_bf16_2d(const TcState& st, void* out, const void* base, uint64_t inner, uint64_t outer,
+                       uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer);
+
+// ---- tensor-core in-place pass (agzo_rmw_tc.cu)
+bool rmw_tc_eligible(const agzo_layer& a);
+void rmw_tc_shape(const agzo_layer& a, DevLayer* D);       // fills the rtc_* fields except item0 / wmap
+bool rmw_tc_encode_map(const TcState& st, const DevLayer& D, void* host_map);
+cudaError_t rmw_tc_init();
+cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
+                          int max_rp, uint64_t seed, float coef, const float* d_coef, DevStatus* d_status,
+                          int sm_count, cudaStream_t s);
+
 cudaError_t tc_fill_omega(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,
                           uint64_t seed, cudaStream_t s);
 cudaError_t tc_xt_t(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,

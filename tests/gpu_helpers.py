@@ -55,13 +55,30 @@ def projector_distance(Va: np.ndarray, Vb: np.ndarray) -> float:
     return float(np.sqrt(max(a + b - 2 * c, 0.0)))
 
 
-def cancellation_floor(w_in: np.ndarray, coef: float, seed: int, layer_id: int, V: np.ndarray):
-    """fp32 rounding noise of the operands of w + c*(G V^T): 2^-20 * max(|w|, |c| |G||V|).
-    Where the sum cancels, the result's own ulp is smaller than this noise, so no fp32
-    evaluation can match an exact one to an ulp of the result there."""
+def cancellation_floor(w_in: np.ndarray, coef: float, seed: int, layer_id: int, V: np.ndarray,
+                       rel: float = 2.0 ** -20):
+    """Rounding noise of the operands of w + c*(G V^T): rel * max(|w|, |c| |G||V|).
+    Where the sum cancels, the result's own ulp is smaller than this noise, so no finite
+    precision evaluation can match an exact one to an ulp of the result there.
+    rel = 2^-20 for the CUDA-core kernels (fp32 FMA chain over r terms); 2^-16 for the
+    tensor-core kernel, whose factors are hi + lo bf16 pairs (each carries 2^-18 of its value
+    as residual, two factors per product, one binade of slack)."""
     G = np.abs(O.gen_G(seed, layer_id, w_in.shape[0], V.shape[0]).astype(np.float64))
     A = abs(float(coef)) * (G @ np.abs(V.astype(np.float64)))
-    return 2.0 ** -20 * np.maximum(np.abs(w_in.astype(np.float64)), A)
+    return rel * np.maximum(np.abs(w_in.astype(np.float64)), A)
+
+
+def tc_mismatch_bound(want: np.ndarray, coef: float, seed: int, layer_id: int, V: np.ndarray) -> float:
+    """Share of bf16 results that may land on the neighbouring grid point under the tensor-core
+    kernel.  Its factors are hi + lo bf16 pairs, so c*z carries an absolute error up to
+    e_ij = 2^-17 |c| (|G||V|)_ij (2^-18 of each factor, two factors); a result within e_ij of a
+    rounding boundary can round the other way, which has probability 2 e_ij / ulp(w'_ij).
+    The bound is the mean of that over the matrix (never below the 1e-3 of the other kernels)."""
+    G = np.abs(O.gen_G(seed, layer_id, want.shape[0], V.shape[0]).astype(np.float64))
+    e = 2.0 ** -17 * abs(float(coef)) * (G @ np.abs(V.astype(np.float64)))
+    mag = np.maximum(np.abs(want.astype(np.float64)), 2.0 ** -126)
+    ulp = 2.0 ** (np.floor(np.log2(mag)) - 7)
+    return max(1e-3, float(np.minimum(1.0, 2.0 * e / ulp).mean()))
 
 
 def assert_weights_match(got: np.ndarray, want: np.ndarray, storage: str, frac: float = 1e-3,
