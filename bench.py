@@ -180,6 +180,10 @@ def main():
     ap.add_argument("--rank", type=int, default=16)
     ap.add_argument("--extract-path", type=int, default=0)
     ap.add_argument("--wave-mb", type=int, default=-1)
+    ap.add_argument("--rmw-path", type=int, default=0)
+    ap.add_argument("--rmw-slots", type=int, default=0)
+    ap.add_argument("--rmw-inflight", type=int, default=0)
+    ap.add_argument("--rmw-panels", type=int, default=0)
     ap.add_argument("--blocks", type=int, default=0,
                     help="keep only the first N transformer blocks of the layer set (profiling-sized runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -213,6 +217,10 @@ def main():
     arr = B.layer_array(layers)
     ctx = B.agzo_create(layers, local)
     B.agzo_set_option(ctx, "extract_path", args.extract_path)
+    B.agzo_set_option(ctx, "rmw_path", args.rmw_path)
+    B.agzo_set_option(ctx, "rmw_tc_slots", args.rmw_slots)
+    B.agzo_set_option(ctx, "rmw_tc_inflight", args.rmw_inflight)
+    B.agzo_set_option(ctx, "rmw_tc_panels", args.rmw_panels)
     if args.wave_mb >= 0:
         B.agzo_set_option(ctx, "wave_bytes", args.wave_mb << 20)
     work = algorithmic_work(cfg, r)

@@ -123,7 +123,9 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * "rmw_path" selects the kernel of the in-place passes: 0 = automatic (bf16 weights with
  * 16-byte aligned rows and r >= "rmw_tc_min_rank", default 8, take the tensor-core kernel,
  * everything else the CUDA-core kernels), 1 = CUDA-core kernels only, 2 = tensor-core kernel
- * for every layer that allows it;
+ * for every layer that allows it; tuning knobs of that kernel, 0 = chosen by rank:
+ * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),
+ * "rmw_tc_panels" (column panels per work item, 1 or 2);
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
  * "time_kernel_class" = one agzo_kernel_class whose launches get a CUDA event pair on the
  * caller's stream (0 = none), read back by agzo_read_counters.                           */

@@ -40,6 +40,7 @@ struct PlanOpts {
   int extract_path;      // 0 auto, 1 CUDA-core only, 2 tensor-core required
   int rmw_path;          // 0 auto, 1 CUDA-core only, 2 tensor cores wherever a layer allows it
   int rmw_tc_min_rank;   // auto: layers with r >= this use the tensor-core pass
+  int rmw_tc_panels;     // column panels per work item of the tensor-core pass (1 or 2)
   bool tc_available;
 };
 
@@ -55,6 +56,9 @@ struct agzo_ctx {
   int extract_path;        // 0 auto, 1 CUDA-core only, 2 tensor-core required
   int rmw_path;            // 0 auto, 1 CUDA-core only, 2 tensor cores wherever possible
   int rmw_tc_min_rank;
+  int rmw_tc_slots;        // ring slots of the tensor-core pass, 0 = as many as fit
+  int rmw_tc_inflight;     // loads in flight per CTA, 0 = by rank
+  int rmw_tc_panels;       // column panels per work item (1 or 2), 0 = by rank
   int64_t wave_bytes;
   // descriptors last uploaded
   std::vector<agzo_layer> cached;
@@ -228,7 +232,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
                         (opts.rmw_path == 2 || a.r >= opts.rmw_tc_min_rank);
     plan->item_start[i] = (int)items;
     if (tc_rmw) {
-      rmw_tc_shape(a, &D);
+      rmw_tc_shape(a, opts.rmw_tc_panels, &D);
       D.rtc_item0 = (int)items;
       items += (long long)D.rtc_panels * D.rtc_chunks;
       if (items > 0x7fffffff) return AGZO_ERR_INVALID_ARG;
@@ -318,7 +322,8 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (same_layers(c, L, n)) return AGZO_OK;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
-  const PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->tc.available};
+  const PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels,
+                      c->tc.available};
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st != AGZO_OK) return st;
   const size_t lb = align_up((size_t)n * sizeof(DevLayer));
@@ -375,8 +380,8 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   if (st != AGZO_OK) return st;
   if (c->plan.total_items > 0) {
     Timed t(c, AGZO_KC_RMW_TC, s);
-    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, seed, coef,
-                        d_coef, dev_status(c), c->sm_count, s));
+    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->rmw_tc_slots, c->rmw_tc_inflight, seed,
+                        coef, d_coef, dev_status(c), c->sm_count, s));
   }
   if (c->plan.total_tiles > 0) {
     Timed t(c, AGZO_KC_RMW, s);
@@ -417,9 +422,9 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, true}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, false}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -445,6 +450,9 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->extract_path = 0;
   c->rmw_path = 0;
   c->rmw_tc_min_rank = 8;
+  c->rmw_tc_slots = 0;
+  c->rmw_tc_inflight = 0;
+  c->rmw_tc_panels = 0;
   c->wave_bytes = kDefaultWaveBytes;
   c->cached_valid = false;
   c->h_stage = nullptr;
@@ -492,6 +500,17 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
   } else if (std::strcmp(name, "rmw_tc_min_rank") == 0) {
     if (value < 1 || value > AGZO_MAX_RANK) return AGZO_ERR_INVALID_ARG;
     ctx->rmw_tc_min_rank = (int)value;
+  } else if (std::strcmp(name, "rmw_tc_inflight") == 0) {
+    if (value < 0 || value > 64) return AGZO_ERR_INVALID_ARG;
+    ctx->rmw_tc_inflight = (int)value;
+    return AGZO_OK;
+  } else if (std::strcmp(name, "rmw_tc_panels") == 0) {
+    if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
+    ctx->rmw_tc_panels = (int)value;
+  } else if (std::strcmp(name, "rmw_tc_slots") == 0) {
+    if (value < 0 || value > 64) return AGZO_ERR_INVALID_ARG;
+    ctx->rmw_tc_slots = (int)value;
+    return AGZO_OK;
   } else if (std::strcmp(name, "wave_bytes") == 0) {
     if (value < 0) return AGZO_ERR_INVALID_ARG;
     ctx->wave_bytes = value;

@@ -39,9 +39,10 @@ struct alignas(16) DevLayer {
   long long m_pad;       // row pitch of Tb in elements (m rounded up to 8)
   int NB, NP;
   // tensor-core in-place pass (bf16 W): this layer's work items are
-  // [rtc_item0, rtc_item0 + rtc_panels * rtc_chunks); item = (row chunk, column panel)
+  // [rtc_item0, rtc_item0 + rtc_panels * rtc_chunks); item = (row chunk, group of column panels)
   const void* wmap;      // 128-byte TMA descriptor of W, box = 64 columns x 128 rows; null = CUDA-core pass
-  int rtc_item0, rtc_panels, rtc_chunks;
+  int rtc_item0, rtc_panels, rtc_chunks;   // rtc_panels counts panel GROUPS of rtc_np panels
+  int rtc_np;            // column panels per item (they share the R operand of a row tile)
   int rtc_chunk_blocks;  // 128-row blocks per row chunk
   int rtc_cw;            // columns per panel: 256, 128 or 64
   int rtc_rp;            // rank rounded up to a multiple of 8

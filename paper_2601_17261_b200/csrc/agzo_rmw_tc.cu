@@ -11,9 +11,13 @@
 // are laid side by side along K (K index = [RhAh | RhAl | RlAh | RlAl]), so the products are
 // exact and summed in fp32; what is dropped is below 2^-17 of each term.
 //
+// Work item = (layer, chunk of up to 8 row tiles, group of up to two adjacent column panels).
+// The R operand of a row tile serves every panel of the group, so R is regenerated once per
+// 128 x (2 * panel width) weights and the CTA streams up to 1 KiB of every weight row.
+//
 // Data flow of one CTA (persistent, one per SM):
 //   loader thread      TMA-loads 128 x 64 boxes of W into a ring of shared-memory slots
-//   R warps (4)        regenerate the tile's 128 rows of R from the Philox counter and write the
+//   R warps (4 or 8)   regenerate the tile's 128 rows of R from the Philox counter and write the
 //                      split A operand; at the start of an item they also build the B operand
 //                      from the panel's slice of A^T (V)
 //   MMA thread         issues the tcgen05.mma chain into one of two TMEM buffers
@@ -37,11 +41,12 @@ constexpr int kRows = 128;                 // rows of a tile (MMA M)
 constexpr int kBoxCols = 64;               // columns of one W box = one 128-byte swizzle row
 constexpr int kBoxBytes = kRows * 128;     // 16 KiB
 constexpr int kAtomBytesA = kRows * 128;   // one 64-wide K atom of the A operand
-constexpr int kBBytes = 32 * 1024;         // B operand: panel columns x K, always 32 KiB
+constexpr int kBBytes = 32 * 1024;         // B operand of one panel: panel columns x K, always 32 KiB
+constexpr int kMaxPanels = 2;              // panels per work item
 constexpr int kMaxSlots = 12;
 constexpr int kWarpLoader = 0, kWarpMma = 1, kWarpStorer = 2, kWarpEpi0 = 3, kNumEpiWarps = 8,
-              kWarpGen0 = kWarpEpi0 + kNumEpiWarps, kNumGenWarps = 4;
-constexpr int kThreads = (kWarpGen0 + kNumGenWarps) * 32;   // 480
+              kWarpGen0 = kWarpEpi0 + kNumEpiWarps, kMaxGenWarps = 8;
+constexpr int kMaxThreads = (kWarpGen0 + kMaxGenWarps) * 32;   // 608
 constexpr uint32_t kTmemCols = 512;        // two delta buffers of up to 256 columns
 
 struct Shared {
@@ -57,7 +62,13 @@ struct Shared {
 
 struct Item {
   const DevLayer* L;
-  int col0, rb0, rb1, cw, rp, nboxes;
+  int col0, rb0, rb1, cw, rp, np;   // np = live panels of the group (1 or 2)
+  __device__ __forceinline__ int panel_col(int p) const { return col0 + p * cw; }
+  __device__ __forceinline__ int nboxes(int p) const {   // boxes of panel p that hold columns of W
+    const int left = L_d_in - panel_col(p);
+    return min(cw / kBoxCols, (left + kBoxCols - 1) / kBoxCols);
+  }
+  int L_d_in;
 };
 
 __device__ __forceinline__ int find_layer_of_item(const int* start, int n_layers, int item) {
@@ -73,16 +84,16 @@ __device__ __forceinline__ Item decode_item(const DevLayer* layers, const int* i
   Item it;
   const DevLayer* L = layers + find_layer_of_item(item_start, n_layers, item);
   it.L = L;
+  it.L_d_in = L->d_in;
   const int local = item - L->rtc_item0;
-  const int chunk = local / L->rtc_panels, panel = local - chunk * L->rtc_panels;
+  const int chunk = local / L->rtc_panels, group = local - chunk * L->rtc_panels;
   it.cw = L->rtc_cw;
   it.rp = L->rtc_rp;
-  it.col0 = panel * it.cw;
+  it.col0 = group * L->rtc_np * it.cw;
   const int nrb = (L->d_out + kRows - 1) / kRows;
   it.rb0 = chunk * L->rtc_chunk_blocks;
   it.rb1 = min(nrb, it.rb0 + L->rtc_chunk_blocks);
-  const int cols_left = L->d_in - it.col0;
-  it.nboxes = min(it.cw / kBoxCols, (cols_left + kBoxCols - 1) / kBoxCols);
+  it.np = min(L->rtc_np, (L->d_in - it.col0 + it.cw - 1) / it.cw);
   return it;
 }
 
@@ -117,21 +128,19 @@ __device__ __forceinline__ void put_group(uint8_t* base, int atom_bytes, int row
   }
 }
 
-__device__ __forceinline__ float pick(const float4& g, int lane) {
-  return lane == 0 ? g.x : lane == 1 ? g.y : lane == 2 ? g.z : g.w;
-}
-
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMaxThreads, 1)
 rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_start, int n_layers,
-              int total_items, int a_bufs, int a_buf_bytes, int slots, uint64_t seed, float coef_imm,
+              int total_items, int a_bufs, int a_buf_bytes, int slots, int inflight, uint64_t seed, float coef_imm,
               const float* __restrict__ d_coef, DevStatus* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = base;                                   // a_bufs x a_buf_bytes
-  uint8_t* sB = sA + (size_t)a_bufs * a_buf_bytes;      // kBBytes
-  uint8_t* sW = sB + kBBytes;                           // slots x kBoxBytes
+  uint8_t* sB = sA + (size_t)a_bufs * a_buf_bytes;      // kMaxPanels x kBBytes
+  uint8_t* sW = sB + kMaxPanels * kBBytes;              // slots x kBoxBytes
   __shared__ Shared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gen_warps = (int)(blockDim.x >> 5) - kWarpGen0;   // 4 for small ranks, 8 otherwise
+  const int gen_threads = gen_warps * 32;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < slots; ++s) {
@@ -140,12 +149,12 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
       mbar_init(&sh.empty_w[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&sh.a_full[b], kNumGenWarps);
+      mbar_init(&sh.a_full[b], gen_warps);
       mbar_init(&sh.a_empty[b], 1);
       mbar_init(&sh.tmem_full[b], 1);
       mbar_init(&sh.tmem_empty[b], kNumEpiWarps);
     }
-    mbar_init(&sh.b_full, kNumGenWarps);
+    mbar_init(&sh.b_full, gen_warps);
     mbar_init(&sh.b_empty, 1);
     sh.failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -166,11 +175,18 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
         const void* map = it.L->wmap;
         tmap_acquire(map);
         for (int rb = it.rb0; rb < it.rb1 && ok; ++rb) {
-          for (int j = 0; j < it.nboxes; ++j, ++n) {
-            const int s = n % slots, u = n / slots;
-            if (u > 0 && !mbar_wait(&sh.empty_w[s], (u - 1) & 1)) { ok = false; break; }
-            mbar_expect_tx(&sh.full_w[s], kBoxBytes);
-            tma_load_2d(sW + (size_t)s * kBoxBytes, map, it.col0 + j * kBoxCols, rb * kRows, &sh.full_w[s]);
+          for (int p = 0; p < it.np && ok; ++p) {
+            const int nb = it.nboxes(p), pc = it.panel_col(p);
+            for (int j = 0; j < nb; ++j, ++n) {
+              const int s = n % slots, u = n / slots;
+              if (u > 0 && !mbar_wait(&sh.empty_w[s], (u - 1) & 1)) { ok = false; break; }
+              if (n >= inflight) {              // at most `inflight` loads outstanding: box n - inflight has landed
+                const int k = n - inflight;
+                if (!mbar_wait(&sh.full_w[k % slots], (k / slots) & 1)) { ok = false; break; }
+              }
+              mbar_expect_tx(&sh.full_w[s], kBoxBytes);
+              tma_load_2d(sW + (size_t)s * kBoxBytes, map, pc + j * kBoxCols, rb * kRows, &sh.full_w[s]);
+            }
           }
         }
       }
@@ -188,14 +204,17 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
         const void* map = it.L->wmap;
         tmap_acquire(map);
         for (int rb = it.rb0; rb < it.rb1 && ok; ++rb) {
-          for (int j = 0; j < it.nboxes; ++j, ++n) {
-            const int s = n % slots, u = n / slots;
-            if (!mbar_wait(&sh.epi_done[s], u & 1)) { ok = false; break; }
-            tma_store_2d(map, it.col0 + j * kBoxCols, rb * kRows, sW + (size_t)s * kBoxBytes);
-            tma_commit_group();
-            if (n > 0) {                      // the previous box's store has read its slot
-              tma_wait_group_read<1>();
-              mbar_arrive(&sh.empty_w[(n - 1) % slots]);
+          for (int p = 0; p < it.np && ok; ++p) {
+            const int nb = it.nboxes(p), pc = it.panel_col(p);
+            for (int j = 0; j < nb; ++j, ++n) {
+              const int s = n % slots, u = n / slots;
+              if (!mbar_wait(&sh.epi_done[s], u & 1)) { ok = false; break; }
+              tma_store_2d(map, pc + j * kBoxCols, rb * kRows, sW + (size_t)s * kBoxBytes);
+              tma_commit_group();
+              if (n > 0) {                      // the previous box's store has read its slot
+                tma_wait_group_read<1>();
+                mbar_arrive(&sh.empty_w[(n - 1) % slots]);
+              }
             }
           }
         }
@@ -205,7 +224,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
     }
   } else if (warp == kWarpMma) {
     if (lane == 0) {
-      int t = 0, ic = 0;
+      int t = 0, ta = 0, ic = 0;      // t counts (row tile, panel) pairs, ta row tiles, ic items
       bool ok = true;
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++ic) {
         const Item it = decode_item(layers, item_start, n_layers, item);
@@ -213,29 +232,33 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
         const uint32_t idesc = instr_desc(kRows, it.cw, 0, 0);
         const int ksteps = it.rp / 4;                    // K = 4 * rp, 16 per instruction
         const uint32_t b_atom = (uint32_t)it.cw * 128u;
-        for (int rb = it.rb0; rb < it.rb1; ++rb, ++t) {
-          const int ab = t % a_bufs, au = t / a_bufs;
+        for (int rb = it.rb0; rb < it.rb1 && ok; ++rb, ++ta) {
+          const int ab = ta % a_bufs, au = ta / a_bufs;
           if (!mbar_wait(&sh.a_full[ab], au & 1)) { ok = false; break; }
-          const int tb = t & 1, tu = t >> 1;
-          if (tu > 0 && !mbar_wait(&sh.tmem_empty[tb], (tu - 1) & 1)) { ok = false; break; }
-          tc_fence_after();
           const uint32_t a0 = smem_u32(sA + (size_t)ab * a_buf_bytes);
-          const uint32_t b0 = smem_u32(sB);
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const int ka = ks >> 2, kk = ks & 3;
-            const uint64_t ad = smem_desc(a0 + ka * kAtomBytesA + kk * 32, 0, 1024);
-            const uint64_t bd = smem_desc(b0 + ka * b_atom + kk * 32, 0, 1024);
-            mma_bf16(tmem + (uint32_t)tb * 256u, ad, bd, idesc, ks > 0 ? 1u : 0u);
+          for (int p = 0; p < it.np; ++p, ++t) {
+            const int tb = t & 1, tu = t >> 1;
+            if (tu > 0 && !mbar_wait(&sh.tmem_empty[tb], (tu - 1) & 1)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t b0 = smem_u32(sB + (size_t)p * kBBytes);
+            for (int ks = 0; ks < ksteps; ++ks) {
+              const int ka = ks >> 2, kk = ks & 3;
+              const uint64_t ad = smem_desc(a0 + ka * kAtomBytesA + kk * 32, 0, 1024);
+              const uint64_t bd = smem_desc(b0 + ka * b_atom + kk * 32, 0, 1024);
+              mma_bf16(tmem + (uint32_t)tb * 256u, ad, bd, idesc, ks > 0 ? 1u : 0u);
+            }
+            mma_commit(&sh.tmem_full[tb]);
           }
-          mma_commit(&sh.a_empty[ab]);
-          mma_commit(&sh.tmem_full[tb]);
+          mma_commit(&sh.a_empty[ab]);      // the row tile's R operand has served all its panels
         }
         mma_commit(&sh.b_empty);
       }
       if (!ok) sh.failed = 1;
     }
   } else if (warp >= kWarpGen0) {
-    // ------------------------------------------------ operand builders: thread gt = row of the tile
+    // ------------------------------------------------ operand builders
+    // A unit of work is (operand row, group of 8 rank indices): consecutive threads take
+    // consecutive rows, so every thread has one or two short independent chains to run.
     const int gt = threadIdx.x - kWarpGen0 * 32;
     int t = 0, ic = 0;
     bool ok = true;
@@ -250,19 +273,20 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
         if (!ok) break;
       }
       const int b_atom = it.cw * 128;
-      for (int n = gt; n < it.cw; n += kNumGenWarps * 32) {
-        const int col = it.col0 + n;
-        for (int g = 0; g < g8; ++g) {
-          float v[8];
+      const int ncols = it.np * it.cw;                   // columns of the whole group
+      for (int unit = gt; unit < ncols * g8; unit += gen_threads) {
+        const int g = unit / ncols, nn = unit - g * ncols;
+        const int p = nn / it.cw, n = nn - p * it.cw;
+        const int col = it.col0 + nn;
+        float v[8];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int k = 8 * g + u;
-            v[u] = (k < r && col < L.d_in) ? __ldg(L.V + (long long)k * L.ldv + col) : 0.f;
-          }
-          uint4 hi, lo;
-          split8(v, &hi, &lo);
-          put_group(sB, b_atom, n, g, g8, hi, lo, 0, 2, 1, 3);
+        for (int u = 0; u < 8; ++u) {
+          const int k = 8 * g + u;
+          v[u] = (k < r && col < L.d_in) ? __ldg(L.V + (long long)k * L.ldv + col) : 0.f;
         }
+        uint4 hi, lo;
+        split8(v, &hi, &lo);
+        put_group(sB + (size_t)p * kBBytes, b_atom, n, g, g8, hi, lo, 0, 2, 1, 3);
       }
       fence_proxy_async();
       __syncwarp();
@@ -276,30 +300,36 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
           if (!ok) break;
         }
         uint8_t* a_base = sA + (size_t)ab * a_buf_bytes;
-        const long long row = (long long)rb * kRows + gt;
-        const bool live = row < L.d_out;
-        const long long e0 = row * r;
-        long long cur = -1;
-        float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int g = 0; g < g8; ++g) {
+        for (int unit = gt; unit < kRows * g8; unit += gen_threads) {
+          const int g = unit >> 7, i = unit & (kRows - 1);
+          const long long row = (long long)rb * kRows + i;
+          const int nv = row < L.d_out ? min(8, r - 8 * g) : 0;   // live rank indices of this group
           float v[8];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int k = 8 * g + u;
-            float x = 0.f;
-            if (live && k < r) {
-              const long long e = e0 + k;
-              if ((e >> 2) != cur) {
-                cur = e >> 2;
-                g4 = gaussian_block((uint64_t)cur, L.layer_id, kTagG, seed);
-              }
-              x = pick(g4, (int)(e & 3));
+          for (int u = 0; u < 8; ++u) v[u] = 0.f;
+          if (nv > 0) {
+            // elements e_first .. e_first + nv - 1 of the stream: at most three Philox blocks
+            const long long e_first = row * r + 8 * g;
+            const long long b0 = e_first >> 2;
+            const int off = (int)(e_first & 3);
+            const int nblk = (off + nv + 3) >> 2;
+            float x[12];
+            const float4 ga = gaussian_block((uint64_t)b0, L.layer_id, kTagG, seed);
+            x[0] = ga.x; x[1] = ga.y; x[2] = ga.z; x[3] = ga.w;
+            float4 gb = make_float4(0.f, 0.f, 0.f, 0.f), gc = gb;
+            if (nblk > 1) gb = gaussian_block((uint64_t)(b0 + 1), L.layer_id, kTagG, seed);
+            if (nblk > 2) gc = gaussian_block((uint64_t)(b0 + 2), L.layer_id, kTagG, seed);
+            x[4] = gb.x; x[5] = gb.y; x[6] = gb.z; x[7] = gb.w;
+            x[8] = gc.x; x[9] = gc.y; x[10] = gc.z; x[11] = gc.w;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float y = off == 0 ? x[u] : off == 1 ? x[u + 1] : off == 2 ? x[u + 2] : x[u + 3];
+              v[u] = u < nv ? y : 0.f;
             }
-            v[u] = x;
           }
           uint4 hi, lo;
           split8(v, &hi, &lo);
-          put_group(a_base, kAtomBytesA, gt, g, g8, hi, lo, 0, 1, 2, 3);
+          put_group(a_base, kAtomBytesA, i, g, g8, hi, lo, 0, 1, 2, 3);
         }
         fence_proxy_async();
         __syncwarp();
@@ -314,27 +344,31 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
     const int h = e >> 2;              // which half of a box's 64 columns
     const int i = q * 32 + lane;       // row inside the tile
     const float coef = d_coef ? __ldg(d_coef) : coef_imm;
-    int t = 0, n = 0;
+    uint32_t off[4];                   // this thread's four 16-byte chunks inside any box
+#pragma unroll
+    for (int c = 0; c < 4; ++c) off[c] = swz(i, h * 4 + c);
+    const uint32_t tmem_row = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 32);
+    int t = 0, s = 0, u = 0;           // tile counter; ring slot and how often the ring has wrapped
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
       const Item it = decode_item(layers, item_start, n_layers, item);
-      for (int rb = it.rb0; rb < it.rb1 && ok; ++rb, ++t) {
+      for (int rbp = it.rb0 * it.np; rbp < it.rb1 * it.np && ok; ++rbp, ++t) {   // (row tile, panel) pairs
         const int tb = t & 1, tu = t >> 1;
         ok = mbar_wait(&sh.tmem_full[tb], tu & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        for (int j = 0; j < it.nboxes; ++j, ++n) {
-          const int s = n % slots, u = n / slots;
+        const int nb = it.nboxes(rbp % it.np);
+        for (int j = 0; j < nb; ++j) {
           ok = mbar_wait(&sh.full_w[s], u & 1);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           uint32_t z[32];
-          tmem_ld32_issue(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * 256 + j * kBoxCols + h * 32), z);
+          tmem_ld32_issue(tmem_row + (uint32_t)(tb * 256 + j * kBoxCols), z);
           uint8_t* slot = sW + (size_t)s * kBoxBytes;
           uint4 w[4];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) w[c] = *reinterpret_cast<const uint4*>(slot + swz(i, h * 4 + c));
+          for (int c = 0; c < 4; ++c) w[c] = *reinterpret_cast<const uint4*>(slot + off[c]);
           tmem_ld_wait();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -347,11 +381,12 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
               const float o1 = fmaf(coef, __uint_as_float(z[8 * c + 2 * p + 1]), w1);
               o[p] = pack2(o0, o1);
             }
-            *reinterpret_cast<uint4*>(slot + swz(i, h * 4 + c)) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(slot + off[c]) = make_uint4(o[0], o[1], o[2], o[3]);
           }
           fence_proxy_async();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.epi_done[s]);
+          if (++s == slots) { s = 0; u ^= 1; }
         }
         tc_fence_before();
         __syncwarp();
@@ -374,13 +409,18 @@ bool rmw_tc_eligible(const agzo_layer& a) {
          (a.ldw * 2) % 16 == 0 && a.d_out >= 1 && a.d_in >= 1 && a.r >= 1 && a.r <= AGZO_MAX_RANK;
 }
 
-void rmw_tc_shape(const agzo_layer& a, DevLayer* D) {
+void rmw_tc_shape(const agzo_layer& a, int panels, DevLayer* D) {
   const int rp = (a.r + 7) & ~7;
   const int katoms = (4 * rp + 63) / 64;                 // 1, 2, 3 or 4 K atoms of 64
   const int cw = katoms == 1 ? 256 : katoms == 2 ? 128 : 64;
+  // panels == 0: one panel per item while R is cheap to regenerate (rp <= 16: the pass is
+  // HBM-bound either way and the smaller items balance better), two from there on, where
+  // regenerating R is what limits the pass
+  const int np = panels == 1 ? 1 : panels == 2 ? kMaxPanels : (katoms == 1 ? 1 : kMaxPanels);
   D->rtc_rp = rp;
   D->rtc_cw = cw;
-  D->rtc_panels = (a.d_in + cw - 1) / cw;
+  D->rtc_np = np;
+  D->rtc_panels = (a.d_in + np * cw - 1) / (np * cw);   // panel groups
   D->rtc_chunk_blocks = 8;
   const int nrb = (a.d_out + kRows - 1) / kRows;
   D->rtc_chunks = (nrb + D->rtc_chunk_blocks - 1) / D->rtc_chunk_blocks;
@@ -397,19 +437,26 @@ cudaError_t rmw_tc_init() {
 }
 
 cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
-                          int max_rp, uint64_t seed, float coef, const float* d_coef, DevStatus* d_status,
-                          int sm_count, cudaStream_t s) {
+                          int max_rp, int slots_wanted, int inflight, uint64_t seed, float coef, const float* d_coef,
+                          DevStatus* d_status, int sm_count, cudaStream_t s) {
   if (total_items <= 0) return cudaSuccess;
   const int katoms = (4 * max_rp + 63) / 64;
   const int a_buf_bytes = katoms * kAtomBytesA;
   const int a_bufs = katoms >= 3 ? 1 : 2;
-  const int fixed = a_bufs * a_buf_bytes + kBBytes;
+  const int fixed = a_bufs * a_buf_bytes + kMaxPanels * kBBytes;
   int slots = (224 * 1024 - fixed) / kBoxBytes;
   if (slots > kMaxSlots) slots = kMaxSlots;
+  if (slots_wanted >= 2 && slots_wanted < slots) slots = slots_wanted;
   const size_t smem = (size_t)fixed + (size_t)slots * kBoxBytes + 1024;
   const int grid = total_items < sm_count ? total_items : sm_count;
-  rmw_tc_kernel<<<grid, kThreads, smem, s>>>(d_layers, d_item_start, n_layers, total_items, a_bufs, a_buf_bytes,
-                                             slots, seed, coef, d_coef, d_status);
+  // operand-builder warps: four keep up with the stream for rp = 8, larger ranks get eight
+  const int threads = (kWarpGen0 + (max_rp <= 8 ? 4 : kMaxGenWarps)) * 32;
+  // loads in flight per CTA: enough to cover the HBM latency at this SM's share of the
+  // bandwidth (4 to 5 boxes of 16 KiB); more only lengthens the queues in front of the stores
+  if (inflight < 1) inflight = max_rp <= 8 ? 4 : 5;
+  if (inflight > slots) inflight = slots;
+  rmw_tc_kernel<<<grid, threads, smem, s>>>(d_layers, d_item_start, n_layers, total_items, a_bufs, a_buf_bytes,
+                                             slots, inflight, seed, coef, d_coef, d_status);
   return cudaGetLastError();
 }
 
