@@ -31,6 +31,10 @@ import torch  # noqa: E402
 from paper_2601_17261_b200 import workloads as WL  # noqa: E402
 
 K_POWER = 3
+# DRAM bytes moved per algorithmic byte, from the ncu capture of each kernel on a 2-block
+# slice of the 8B-shaped layer set (summaries under profiles/); traffic grows in proportion
+# to the activation bytes a launch sweeps.  Reset an entry to None when its kernel changes.
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (2.430710 + 0.038939) / 2.415919}
 EPS = 1e-3
 LR = 1e-6
 METRIC = "agzo_step_overhead_ms"
@@ -169,6 +173,20 @@ def run_reference(args, cfg, rank_r):
     return 0
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """A timing is the slowest rank's: all-reduce MAX of the per-rank milliseconds (no-op for one rank)."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t)
+
+
+def whole_job_units(per_rank_units: float, world: int) -> float:
+    """Replicas (weak scaling): every rank does the same per-rank work, the job does world times it."""
+    return per_rank_units * world
+
+
 # ----------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -180,6 +198,7 @@ def main():
     ap.add_argument("--rank", type=int, default=16)
     ap.add_argument("--extract-path", type=int, default=0)
     ap.add_argument("--wave-mb", type=int, default=-1)
+    ap.add_argument("--extract-streams", type=int, default=2)
     ap.add_argument("--rmw-path", type=int, default=0)
     ap.add_argument("--rmw-slots", type=int, default=0)
     ap.add_argument("--rmw-inflight", type=int, default=0)
@@ -215,9 +234,11 @@ def main():
 
     Ws, Xs, Vs, layers = build_layer_set(cfg, r, dev)
     arr = B.layer_array(layers)
-    ctx = B.agzo_create(layers, local)
+    # a larger wave than the default needs more scratch than agzo_workspace_bytes reports
+    ctx = B.agzo_create(layers, local, extra_bytes=(12 << 30) if args.wave_mb > 4096 else 0)
     B.agzo_set_option(ctx, "extract_path", args.extract_path)
     B.agzo_set_option(ctx, "rmw_path", args.rmw_path)
+    B.agzo_set_option(ctx, "extract_streams", args.extract_streams)
     B.agzo_set_option(ctx, "rmw_tc_slots", args.rmw_slots)
     B.agzo_set_option(ctx, "rmw_tc_inflight", args.rmw_inflight)
     B.agzo_set_option(ctx, "rmw_tc_panels", args.rmw_panels)
@@ -248,12 +269,7 @@ def main():
             fn(first_seed + i)
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1) / n
-        if dist is not None:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t)
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1) / n, dist, dev)
 
     # ---- warm-up, then the timed region with the dominant kernel class bracketed by events
     for i in range(args.warmup):
@@ -263,13 +279,24 @@ def main():
         raise SystemExit("device status not ok after warm-up")
     tc_used = args.extract_path != 1
     dom_class = B.KC_TC_XT_T if tc_used else B.KC_XT_T
-    B.agzo_set_option(ctx, "time_kernel_class", dom_class)
     B.agzo_read_counters(ctx)
     sampler = ClockSampler(local) if rank == 0 else None
     ms_step = timed(step, args.steps, 100)
     clocks = sampler.stop() if sampler else {}
-    dom_ms, dom_n, launches = B.agzo_read_counters(ctx)
+    _, _, launches = B.agzo_read_counters(ctx)
+
+    # ---- the dominant kernel's own launch duration: the same K steps once more with the
+    # extraction waves on one stream (with two helper streams the kernels of two waves share
+    # the GPU, and a launch's event-to-event time would include its neighbour's work)
+    B.agzo_set_option(ctx, "extract_streams", 1)
+    step(90)
+    B.agzo_set_option(ctx, "time_kernel_class", dom_class)
+    B.agzo_read_counters(ctx)
+    ms_step_one_stream = timed(step, args.steps, 100)
+    dom_ms, dom_n, _ = B.agzo_read_counters(ctx)
     B.agzo_set_option(ctx, "time_kernel_class", 0)
+    B.agzo_set_option(ctx, "extract_streams", args.extract_streams)
+    step(91)
 
     # ---- per-phase timings (outside the timed region), same kernels
     def phase_ms(fn, n=3):
@@ -334,8 +361,13 @@ def main():
                         "GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6},
             "roofline": {"kernel": ("tc_xt_t_kernel" if tc_used else "xt_t_kernel") + " (Y = X^T T)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
-                         "peak_kind": peak_kind, "traffic": None,
-                         "launches": dom_n, "avg_ms": dom_avg_ms},
+                         "peak_kind": peak_kind,
+                         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE["tc_xt_t_kernel"] * x_bytes_per_launch
+                                     if tc_used and dom_n else None),
+                         "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the "
+                                         "first 2 blocks of this workload, scaled by the X bytes a launch reads",
+                         "launches": dom_n, "avg_ms": dom_avg_ms,
+                         "measured_with": "extract_streams=1, %.2f ms per step" % ms_step_one_stream},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }

@@ -127,6 +127,9 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),
  * "rmw_tc_panels" (column panels per work item, 1 or 2);
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
+ * "extract_streams" 2 (default) = alternate waves use two scratch regions and two helper
+ * streams forked from and joined to the caller's stream, so that one wave's short kernels
+ * overlap the other's sweeps over X; 1 = waves strictly one after another;
  * "time_kernel_class" = one agzo_kernel_class whose launches get a CUDA event pair on the
  * caller's stream (0 = none), read back by agzo_read_counters.                           */
 agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value);

@@ -16,7 +16,7 @@ constexpr uint32_t kMagic = 0xA620B200u;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;          // DevStatus + scalar slots
 constexpr size_t kCoefOffset = 64;            // float coefficient slot inside the header
-constexpr int64_t kDefaultWaveBytes = 4ll << 30;
+constexpr int64_t kDefaultWaveBytes = 8ll << 30;
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
@@ -24,6 +24,8 @@ struct Plan {
   std::vector<DevLayer> dev;       // one per layer, scratch pointers filled
   std::vector<int> tile_start;     // n + 1
   std::vector<int> wave_end;       // exclusive end index of each extraction wave
+  std::vector<int> wave_region;    // scratch region (= helper stream) of each wave, -1 = nothing to do
+  int regions = 1;
   int total_tiles = 0;
   int max_r = 0;
   int fast_mode_mask = 0;          // storage modes present among layers on the vector path
@@ -42,6 +44,8 @@ struct PlanOpts {
   int rmw_tc_min_rank;   // auto: layers with r >= this use the tensor-core pass
   int rmw_tc_panels;     // column panels per work item of the tensor-core pass (1 or 2)
   bool tc_available;
+  int extract_regions;   // 1: waves run one after another; 2: alternate waves use two scratch regions
+                         // and two helper streams, so one wave's small kernels overlap the other's sweeps
 };
 
 }  // namespace
@@ -60,6 +64,9 @@ struct agzo_ctx {
   int rmw_tc_inflight;     // loads in flight per CTA, 0 = by rank
   int rmw_tc_panels;       // column panels per work item (1 or 2), 0 = by rank
   int64_t wave_bytes;
+  int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
+  cudaStream_t aux[2];     // helper streams of extraction, forked from and joined to the caller's stream
+  cudaEvent_t fork_ev, join_ev[2];
   // descriptors last uploaded
   std::vector<agzo_layer> cached;
   bool cached_valid;
@@ -200,6 +207,9 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   plan->dev.assign(n, DevLayer{});
   plan->tile_start.assign(n + 1, 0);
   plan->wave_end.clear();
+  plan->wave_region.clear();
+  const int regions = opts.extract_regions == 2 ? 2 : 1;
+  plan->regions = regions;
   plan->max_r = 0;
   plan->fast_mode_mask = 0;
   plan->any_slow = false;
@@ -208,7 +218,9 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   plan->total_items = 0;
   plan->max_rp = 0;
   const size_t base = kHeaderBytes + table_bytes(n);
-  const size_t scratch_cap = ws ? (ws_bytes > base ? ws_bytes - base : 0) : (size_t)-1;
+  const size_t scratch_all = ws ? (ws_bytes > base ? ws_bytes - base : 0) : (size_t)-1;
+  const size_t scratch_cap = ws ? scratch_all / regions / kAlign * kAlign : (size_t)-1;   // per region
+  int real_waves = 0;
   size_t max_wave_scratch = 0;
 
   int tiles = 0;
@@ -259,7 +271,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   // scratch fits the workspace
   int i = 0;
   while (i < n) {
-    if (!has_x(L[i])) { ++i; plan->wave_end.push_back(i); continue; }
+    if (!has_x(L[i])) { ++i; plan->wave_end.push_back(i); plan->wave_region.push_back(-1); continue; }
+    const int region = real_waves++ % regions;
     plan->has_extract = true;
     size_t used = 0;
     int64_t xbytes = 0;
@@ -274,7 +287,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       if (used + need > scratch_cap) return AGZO_ERR_WORKSPACE;
       // carve
       if (ws) {
-        char* p = ws + base + used;
+        char* p = ws + base + (size_t)region * scratch_cap + used;
         DevLayer& D = plan->dev[j];
         const agzo_layer& a = L[j];
         int slabs, slab_rows;
@@ -298,9 +311,10 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
     }
     if (used > max_wave_scratch) max_wave_scratch = used;
     plan->wave_end.push_back(j);
+    plan->wave_region.push_back(region);
     i = j;
   }
-  if (scratch_needed) *scratch_needed = max_wave_scratch;
+  if (scratch_needed) *scratch_needed = max_wave_scratch * regions + (regions > 1 ? kAlign : 0);
   return AGZO_OK;
 }
 
@@ -322,9 +336,13 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (same_layers(c, L, n)) return AGZO_OK;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
-  const PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels,
-                      c->tc.available};
+  PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels,
+                c->tc.available, c->extract_streams};
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
+  if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
+    opts.extract_regions = 1;
+    st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
+  }
   if (st != AGZO_OK) return st;
   const size_t lb = align_up((size_t)n * sizeof(DevLayer));
   const size_t tb = prefix_bytes(n) + (size_t)n * kMapBytes;
@@ -422,9 +440,9 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true, 2}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -454,6 +472,9 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->rmw_tc_inflight = 0;
   c->rmw_tc_panels = 0;
   c->wave_bytes = kDefaultWaveBytes;
+  c->extract_streams = 2;
+  c->aux[0] = c->aux[1] = nullptr;
+  c->fork_ev = c->join_ev[0] = c->join_ev[1] = nullptr;
   c->cached_valid = false;
   c->h_stage = nullptr;
   c->h_stage_bytes = 0;
@@ -465,11 +486,21 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->stage_ev, cudaEventDisableTiming);
+  for (int k = 0; k < 2 && e == cudaSuccess; ++k) {
+    e = cudaStreamCreateWithFlags(&c->aux[k], cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->join_ev[k], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(c->ws, 0, kHeaderBytes);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = tc_init(&c->tc, device);
   if (e != cudaSuccess) {
     if (c->stage_ev) cudaEventDestroy(c->stage_ev);
+    if (c->fork_ev) cudaEventDestroy(c->fork_ev);
+    for (int k = 0; k < 2; ++k) {
+      if (c->join_ev[k]) cudaEventDestroy(c->join_ev[k]);
+      if (c->aux[k]) cudaStreamDestroy(c->aux[k]);
+    }
     delete c;
     return AGZO_ERR_CUDA;
   }
@@ -482,6 +513,12 @@ agzo_status agzo_destroy(agzo_ctx* ctx) {
   if (ctx->stage_pending) cudaEventSynchronize(ctx->stage_ev);
   if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
   if (ctx->stage_ev) cudaEventDestroy(ctx->stage_ev);
+  if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
+  for (int k = 0; k < 2; ++k) {
+    if (ctx->aux[k]) cudaStreamSynchronize(ctx->aux[k]);
+    if (ctx->join_ev[k]) cudaEventDestroy(ctx->join_ev[k]);
+    if (ctx->aux[k]) cudaStreamDestroy(ctx->aux[k]);
+  }
   for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   ctx->magic = 0;
   delete ctx;
@@ -511,6 +548,9 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
     if (value < 0 || value > 64) return AGZO_ERR_INVALID_ARG;
     ctx->rmw_tc_slots = (int)value;
     return AGZO_OK;
+  } else if (std::strcmp(name, "extract_streams") == 0) {
+    if (value < 1 || value > 2) return AGZO_ERR_INVALID_ARG;
+    ctx->extract_streams = (int)value;
   } else if (std::strcmp(name, "wave_bytes") == 0) {
     if (value < 0) return AGZO_ERR_INVALID_ARG;
     ctx->wave_bytes = value;
@@ -572,51 +612,73 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
   if (st != AGZO_OK) return st;
 
   const Plan& P = ctx->plan;
-  int l0 = 0;
-  for (size_t wv = 0; wv < P.wave_end.size(); ++wv) {
-    const int l1 = P.wave_end[wv];
-    ExtractWave w{};
-    w.d_layers = dev_layers(ctx);
-    w.l0 = l0; w.l1 = l1;
-    bool all_tc = ctx->extract_path != 1;
-    for (int i = l0; i < l1; ++i) {
-      const DevLayer& D = P.dev[i];
-      if (D.m > w.max_m) w.max_m = D.m;
-      if (D.d_in > w.max_din) w.max_din = D.d_in;
-      if (D.r > w.max_r) w.max_r = D.r;
-      if (D.slabs > w.max_slabs) w.max_slabs = D.slabs;
-      if (D.gchunks > w.max_gchunks) w.max_gchunks = D.gchunks;
-      if (!D.Qb) all_tc = false;
-    }
-    l0 = l1;
-    if (w.max_m == 0) continue;
-    DevStatus* dst = dev_status(ctx);
-    auto panel_qr = [&]() -> cudaError_t {
-      Timed t(ctx, AGZO_KC_PANEL_QR, s, 3);
-      return launch_panel_qr(w, dst, s);
-    };
-    auto omega = [&]() -> cudaError_t {
-      Timed t(ctx, AGZO_KC_OMEGA, s);
-      return all_tc ? tc_fill_omega(ctx->tc, w, P.dev.data(), seed, s) : launch_fill_omega(w, seed, s);
-    };
-    auto xt_t = [&]() -> cudaError_t {       // Y <- H T
-      Timed t(ctx, all_tc ? AGZO_KC_TC_XT_T : AGZO_KC_XT_T, s);
-      return all_tc ? tc_xt_t(ctx->tc, w, P.dev.data(), dst, s) : launch_xt_t(w, s);
-    };
-    auto x_q = [&]() -> cudaError_t {        // T <- H^T Q
-      Timed t(ctx, all_tc ? AGZO_KC_TC_X_Q : AGZO_KC_X_Q, s);
-      return all_tc ? tc_x_q(ctx->tc, w, P.dev.data(), dst, s) : launch_x_q(w, s);
-    };
-    CU(ctx, omega());                        // Omega
-    CU(ctx, xt_t());                         // Y <- H Omega
-    for (int k = 0; k < K; ++k) {
-      CU(ctx, panel_qr());                   // Q <- qr(Y)
-      CU(ctx, x_q());
-      CU(ctx, xt_t());                       // Y <- H (H^T Q)
-    }
-    CU(ctx, panel_qr());                     // A <- qr(Y)
+  // With two scratch regions, alternate waves run on two helper streams forked from the
+  // caller's stream: the short, latency-bound kernels of one wave (panel QR) overlap the
+  // other wave's sweeps over X.  Everything is joined back before the call returns.
+  int n_real = 0;
+  for (int rg : P.wave_region) n_real += rg >= 0;
+  const bool forked = P.regions == 2 && n_real >= 2;
+  if (forked) {
+    CU(ctx, cudaEventRecord(ctx->fork_ev, s));
+    for (int k = 0; k < 2; ++k) CU(ctx, cudaStreamWaitEvent(ctx->aux[k], ctx->fork_ev, 0));
   }
-  return AGZO_OK;
+  auto run_waves = [&]() -> agzo_status {
+    int l0 = 0;
+    for (size_t wv = 0; wv < P.wave_end.size(); ++wv) {
+      const int l1 = P.wave_end[wv];
+      ExtractWave w{};
+      w.d_layers = dev_layers(ctx);
+      w.l0 = l0; w.l1 = l1;
+      bool all_tc = ctx->extract_path != 1;
+      for (int i = l0; i < l1; ++i) {
+        const DevLayer& D = P.dev[i];
+        if (D.m > w.max_m) w.max_m = D.m;
+        if (D.d_in > w.max_din) w.max_din = D.d_in;
+        if (D.r > w.max_r) w.max_r = D.r;
+        if (D.slabs > w.max_slabs) w.max_slabs = D.slabs;
+        if (D.gchunks > w.max_gchunks) w.max_gchunks = D.gchunks;
+        if (!D.Qb) all_tc = false;
+      }
+      l0 = l1;
+      if (w.max_m == 0 || P.wave_region[wv] < 0) continue;
+      cudaStream_t ws = forked ? ctx->aux[P.wave_region[wv]] : s;
+      DevStatus* dst = dev_status(ctx);
+      auto panel_qr = [&]() -> cudaError_t {
+        Timed t(ctx, AGZO_KC_PANEL_QR, ws, 3);
+        return launch_panel_qr(w, dst, ws);
+      };
+      auto omega = [&]() -> cudaError_t {
+        Timed t(ctx, AGZO_KC_OMEGA, ws);
+        return all_tc ? tc_fill_omega(ctx->tc, w, P.dev.data(), seed, ws) : launch_fill_omega(w, seed, ws);
+      };
+      auto xt_t = [&]() -> cudaError_t {       // Y <- H T
+        Timed t(ctx, all_tc ? AGZO_KC_TC_XT_T : AGZO_KC_XT_T, ws);
+        return all_tc ? tc_xt_t(ctx->tc, w, P.dev.data(), dst, ws) : launch_xt_t(w, ws);
+      };
+      auto x_q = [&]() -> cudaError_t {        // T <- H^T Q
+        Timed t(ctx, all_tc ? AGZO_KC_TC_X_Q : AGZO_KC_X_Q, ws);
+        return all_tc ? tc_x_q(ctx->tc, w, P.dev.data(), dst, ws) : launch_x_q(w, ws);
+      };
+      CU(ctx, omega());                        // Omega
+      CU(ctx, xt_t());                         // Y <- H Omega
+      for (int k = 0; k < K; ++k) {
+        CU(ctx, panel_qr());                   // Q <- qr(Y)
+        CU(ctx, x_q());
+        CU(ctx, xt_t());                       // Y <- H (H^T Q)
+      }
+      CU(ctx, panel_qr());                     // A <- qr(Y)
+    }
+    return AGZO_OK;
+  };
+  st = run_waves();
+  if (forked) {   // join also when a launch failed: the caller's stream must not run ahead of the helpers
+    for (int k = 0; k < 2; ++k) {
+      cudaError_t e = cudaEventRecord(ctx->join_ev[k], ctx->aux[k]);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->join_ev[k], 0);
+      if (e != cudaSuccess && st == AGZO_OK) { ctx->last_cuda = (int)e; st = AGZO_ERR_CUDA; }
+    }
+  }
+  return st;
 }
 
 agzo_status agzo_perturb(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,

@@ -1,0 +1,59 @@
+"""The N > 1 logic of the benchmark on CPU: two gloo ranks.
+
+The hot path has no exchange step (every rank of a zeroth-order data-parallel job holds the
+whole model and applies the same seeded perturbation), so several GPUs run replicas.  What the
+ranks do share is the measurement protocol: a timing is the maximum over ranks, rank 0 alone
+reports, and the reference arm runs on rank 0 only.
+"""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ms = bench.max_over_ranks(10.0 + 5.0 * rank, dist, torch.device("cpu"))
+        out[rank] = ms
+        # every rank regenerates the same direction from the same seed: nothing to exchange
+        from oracle import agzo_oracle as O
+        g = torch.from_numpy(O.gen_G(7, 3, 16, 4).copy())
+        gathered = [torch.zeros_like(g) for _ in range(world)]
+        dist.all_gather(gathered, g)
+        out[world + rank] = all(bool((x == g).all()) for x in gathered)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_timing_is_the_maximum_over_ranks_and_directions_need_no_exchange():
+    world, port = 2, 29611
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+        assert out[0] == out[1] == 15.0
+        assert out[2] and out[3]
+
+
+def test_single_rank_timing_is_passed_through():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(3.25, None, torch.device("cpu")) == 3.25
+    assert bench.whole_job_units(2.0, 4) == 8.0
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0
+    assert not [l for l in p.stdout.splitlines() if l.startswith("{")]
