@@ -199,6 +199,7 @@ def main():
     ap.add_argument("--extract-path", type=int, default=0)
     ap.add_argument("--wave-mb", type=int, default=-1)
     ap.add_argument("--extract-streams", type=int, default=2)
+    ap.add_argument("--extract-fused", type=int, default=0)
     ap.add_argument("--rmw-path", type=int, default=0)
     ap.add_argument("--rmw-slots", type=int, default=0)
     ap.add_argument("--rmw-inflight", type=int, default=0)
@@ -239,6 +240,7 @@ def main():
     B.agzo_set_option(ctx, "extract_path", args.extract_path)
     B.agzo_set_option(ctx, "rmw_path", args.rmw_path)
     B.agzo_set_option(ctx, "extract_streams", args.extract_streams)
+    B.agzo_set_option(ctx, "extract_fused", args.extract_fused)
     B.agzo_set_option(ctx, "rmw_tc_slots", args.rmw_slots)
     B.agzo_set_option(ctx, "rmw_tc_inflight", args.rmw_inflight)
     B.agzo_set_option(ctx, "rmw_tc_panels", args.rmw_panels)

@@ -119,13 +119,16 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
 agzo_status agzo_destroy(agzo_ctx* ctx);
 
 /* Options: "extract_path" 0 = automatic, 1 = CUDA-core fp32 kernels only, 2 = require the
- * tensor-core kernels (UNSUPPORTED at call time if a layer cannot use them);
+ * tensor-core kernels (UNSUPPORTED at call time if a layer cannot use them), 3 = as 2 but
+ * without the fused power-step kernel (T = X Q and Y = X^T T as two sweeps over X);
  * "rmw_path" selects the kernel of the in-place passes: 0 = automatic (bf16 weights with
  * 16-byte aligned rows and r >= "rmw_tc_min_rank", default 8, take the tensor-core kernel,
  * everything else the CUDA-core kernels), 1 = CUDA-core kernels only, 2 = tensor-core kernel
  * for every layer that allows it; tuning knobs of that kernel, 0 = chosen by rank:
  * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),
  * "rmw_tc_panels" (column panels per work item, 1 or 2);
+ * "extract_fused" 1 = layers with r <= 16 and d_in <= 4096 on the tensor-core path run each
+ * power step in the fused kernel that reads X once (thread-block clusters); 0 = off;
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
  * "extract_streams" 2 (default) = alternate waves use two scratch regions and two helper
  * streams forked from and joined to the caller's stream, so that one wave's short kernels
@@ -143,7 +146,8 @@ typedef enum agzo_kernel_class {
   AGZO_KC_TC_XT_T = 5,    /* Y = X^T T, tensor-core kernel                                 */
   AGZO_KC_TC_X_Q = 6,     /* T = X Q, tensor-core kernel                                   */
   AGZO_KC_OMEGA = 7,      /* Gaussian test matrix fill                                     */
-  AGZO_KC_RMW_TC = 8      /* the in-place low-rank pass, tensor-core kernel                */
+  AGZO_KC_RMW_TC = 8,     /* the in-place low-rank pass, tensor-core kernel                */
+  AGZO_KC_FUSED_POWER = 9 /* Y = X^T (X Q) in one pass over X, tensor-core cluster kernel  */
 } agzo_kernel_class;
 
 /* Measurement aid.  Waits for the timed launches recorded since the last read, then returns

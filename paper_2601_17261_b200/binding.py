@@ -33,7 +33,7 @@ EXPORTS = [
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
     "agzo_extract_subspace_static",
 ]
-KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC = 1, 2, 3, 4, 5, 6, 7, 8
+KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC, KC_FUSED_POWER = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 
 class agzo_layer(C.Structure):

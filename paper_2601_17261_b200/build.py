@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libagzo.so")
-SOURCES = ["agzo_api.cu", "agzo_rmw.cu", "agzo_rmw_tc.cu", "agzo_extract.cu", "agzo_extract_tc.cu", "agzo_static.cu"]
+SOURCES = ["agzo_api.cu", "agzo_rmw.cu", "agzo_rmw_tc.cu", "agzo_extract.cu", "agzo_extract_tc.cu", "agzo_extract_fused.cu", "agzo_static.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -44,6 +44,7 @@ struct PlanOpts {
   int rmw_tc_min_rank;   // auto: layers with r >= this use the tensor-core pass
   int rmw_tc_panels;     // column panels per work item of the tensor-core pass (1 or 2)
   bool tc_available;
+  bool extract_fused;    // power steps of eligible layers run in the fused single-pass kernel
   int extract_regions;   // 1: waves run one after another; 2: alternate waves use two scratch regions
                          // and two helper streams, so one wave's small kernels overlap the other's sweeps
 };
@@ -65,6 +66,7 @@ struct agzo_ctx {
   int rmw_tc_panels;       // column panels per work item (1 or 2), 0 = by rank
   int64_t wave_bytes;
   int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
+  int extract_fused;       // 1: fused power-step kernel where a layer's shape allows it
   cudaStream_t aux[2];     // helper streams of extraction, forked from and joined to the caller's stream
   cudaEvent_t fork_ev, join_ev[2];
   // descriptors last uploaded
@@ -303,6 +305,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
         if (tc) {
           tc_carve(a, &D, p);
           D.tmaps = ws + maps_offset(n) + (size_t)j * kMapBytes;
+          // the power steps of this layer run fused (X read once per step) where its shape allows
+          D.fz_C = (opts.extract_fused && extract_path != 3 && fused_eligible(a)) ? fused_cluster_size(a) : 0;
         }
       }
       used += need;
@@ -337,7 +341,7 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
   PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels,
-                c->tc.available, c->extract_streams};
+                c->tc.available, c->extract_fused != 0, c->extract_streams};
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
     opts.extract_regions = 1;
@@ -440,9 +444,9 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true, 2}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true, false, 2}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false, 2}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -473,6 +477,7 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->rmw_tc_panels = 0;
   c->wave_bytes = kDefaultWaveBytes;
   c->extract_streams = 2;
+  c->extract_fused = 0;
   c->aux[0] = c->aux[1] = nullptr;
   c->fork_ev = c->join_ev[0] = c->join_ev[1] = nullptr;
   c->cached_valid = false;
@@ -529,7 +534,7 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
   if (!ctx || ctx->magic != kMagic) return AGZO_ERR_STATE;
   if (!name) return AGZO_ERR_INVALID_ARG;
   if (std::strcmp(name, "extract_path") == 0) {
-    if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
+    if (value < 0 || value > 3) return AGZO_ERR_INVALID_ARG;
     ctx->extract_path = (int)value;
   } else if (std::strcmp(name, "rmw_path") == 0) {
     if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
@@ -548,6 +553,9 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
     if (value < 0 || value > 64) return AGZO_ERR_INVALID_ARG;
     ctx->rmw_tc_slots = (int)value;
     return AGZO_OK;
+  } else if (std::strcmp(name, "extract_fused") == 0) {
+    if (value < 0 || value > 1) return AGZO_ERR_INVALID_ARG;
+    ctx->extract_fused = (int)value;
   } else if (std::strcmp(name, "extract_streams") == 0) {
     if (value < 1 || value > 2) return AGZO_ERR_INVALID_ARG;
     ctx->extract_streams = (int)value;
@@ -555,7 +563,7 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
     if (value < 0) return AGZO_ERR_INVALID_ARG;
     ctx->wave_bytes = value;
   } else if (std::strcmp(name, "time_kernel_class") == 0) {
-    if (value < 0 || value > 8) return AGZO_ERR_INVALID_ARG;
+    if (value < 0 || value > 9) return AGZO_ERR_INVALID_ARG;
     ctx->time_class = (int)value;
     return AGZO_OK;
   } else {
@@ -605,7 +613,7 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
   if (st != AGZO_OK) return st;
   if (n == 0) return AGZO_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (ctx->extract_path == 2)
+  if (ctx->extract_path >= 2)
     for (int i = 0; i < n; ++i)
       if (!ctx->tc.available || !tc_eligible(h_layers[i])) return AGZO_ERR_UNSUPPORTED;
   st = prepare(ctx, h_layers, n, s);
@@ -651,20 +659,38 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
         Timed t(ctx, AGZO_KC_OMEGA, ws);
         return all_tc ? tc_fill_omega(ctx->tc, w, P.dev.data(), seed, ws) : launch_fill_omega(w, seed, ws);
       };
-      auto xt_t = [&]() -> cudaError_t {       // Y <- H T
+      // layers served by the fused power-step kernel, by cluster size; the rest take T = X Q, Y = X^T T
+      unsigned fz_classes = 0;
+      bool any_unfused = false;
+      for (int i = w.l0; i < w.l1; ++i) {
+        if (all_tc && P.dev[i].fz_C) fz_classes |= 1u << P.dev[i].fz_C; else any_unfused = true;
+      }
+      auto xt_t = [&](bool skip_fused) -> cudaError_t {       // Y <- H T
         Timed t(ctx, all_tc ? AGZO_KC_TC_XT_T : AGZO_KC_XT_T, ws);
-        return all_tc ? tc_xt_t(ctx->tc, w, P.dev.data(), dst, ws) : launch_xt_t(w, ws);
+        return all_tc ? tc_xt_t(ctx->tc, w, P.dev.data(), dst, skip_fused, ws) : launch_xt_t(w, ws);
       };
       auto x_q = [&]() -> cudaError_t {        // T <- H^T Q
         Timed t(ctx, all_tc ? AGZO_KC_TC_X_Q : AGZO_KC_X_Q, ws);
-        return all_tc ? tc_x_q(ctx->tc, w, P.dev.data(), dst, ws) : launch_x_q(w, ws);
+        return all_tc ? tc_x_q(ctx->tc, w, P.dev.data(), dst, true, ws) : launch_x_q(w, ws);
+      };
+      auto power_fused = [&]() -> cudaError_t {              // Y <- H (H^T Q) in one pass
+        for (int C = 1; C <= 8; ++C) {
+          if (!(fz_classes & (1u << C))) continue;
+          Timed t(ctx, AGZO_KC_FUSED_POWER, ws);
+          cudaError_t e = launch_fused_power_step(w, P.dev.data(), C, dst, ctx->sm_count, ws);
+          if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
       };
       CU(ctx, omega());                        // Omega
-      CU(ctx, xt_t());                         // Y <- H Omega
+      CU(ctx, xt_t(false));                    // Y <- H Omega
       for (int k = 0; k < K; ++k) {
         CU(ctx, panel_qr());                   // Q <- qr(Y)
-        CU(ctx, x_q());
-        CU(ctx, xt_t());                       // Y <- H (H^T Q)
+        if (fz_classes) CU(ctx, power_fused());
+        if (any_unfused) {
+          CU(ctx, x_q());
+          CU(ctx, xt_t(true));                 // Y <- H (H^T Q)
+        }
       }
       CU(ctx, panel_qr());                     // A <- qr(Y)
     }

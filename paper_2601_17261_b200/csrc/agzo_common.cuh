@@ -38,6 +38,7 @@ struct alignas(16) DevLayer {
   const void* tmaps;     // four 128-byte TMA descriptors of this layer: X, Qb, Tb, unused
   long long m_pad;       // row pitch of Tb in elements (m rounded up to 8)
   int NB, NP;
+  int fz_C;              // cluster size of the fused power-step kernel for this layer, 0 = unfused kernels
   // tensor-core in-place pass (bf16 W): this layer's work items are
   // [rtc_item0, rtc_item0 + rtc_panels * rtc_chunks); item = (row chunk, group of column panels)
   const void* wmap;      // 128-byte TMA descriptor of W, box = 64 columns x 128 rows; null = CUDA-core pass

@@ -55,10 +55,10 @@ __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16* hi, __nv_bflo
 // ---------------------------------------------------------------- T = X Q  (Tt = T^T as bf16 hi/lo)
 // One CTA per 128-token tile of one layer.  grid = (max token tiles, layers in the wave).
 __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __restrict__ layers, int l0,
-                                                            DevStatus* status, int stages) {
+                                                            DevStatus* status, int stages, int skip_fused) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const int t0 = blockIdx.x * 128;
-  if (t0 >= L.m) return;
+  if (t0 >= L.m || (skip_fused && L.fz_C)) return;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ TcShared sh;
@@ -155,11 +155,11 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
 // ---------------------------------------------------------------- Ypart[s] = X_s^T T_s
 // One CTA per (128 columns of X, token slab) of one layer.  grid = (column chunks, slabs, layers).
 __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __restrict__ layers, int l0,
-                                                             DevStatus* status, int stages) {
+                                                             DevStatus* status, int stages, int skip_fused) {
   const DevLayer& L = layers[l0 + blockIdx.z];
   const int d0 = blockIdx.x * 128;
   const int slab = blockIdx.y;
-  if (d0 >= L.d_in || slab >= L.slabs) return;
+  if (d0 >= L.d_in || slab >= L.slabs || (skip_fused && L.fz_C)) return;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ TcShared sh;
@@ -354,6 +354,7 @@ cudaError_t tc_init(TcState* st, int device) {
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(tc_xt_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = rmw_tc_init();
+    if (e == cudaSuccess) e = fused_init();
     if (e != cudaSuccess) { cudaGetLastError(); st->available = false; }
   }
   return cudaSuccess;
@@ -404,22 +405,24 @@ cudaError_t tc_fill_omega(const TcState&, const ExtractWave& w, const DevLayer*,
 }
 
 cudaError_t tc_xt_t(const TcState&, const ExtractWave& w, const DevLayer* h_dev, DevStatus* d_status,
-                    cudaStream_t s) {
+                    bool skip_fused, cudaStream_t s) {
   int max_nb = 0;
   for (int i = w.l0; i < w.l1; ++i) max_nb = h_dev[i].NB > max_nb ? h_dev[i].NB : max_nb;
   const int stages = stages_for(max_nb);
   dim3 grid((w.max_din + 127) / 128, w.max_slabs, w.l1 - w.l0);
-  tc_xt_t_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages);
+  tc_xt_t_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages,
+                                                                    skip_fused ? 1 : 0);
   return cudaGetLastError();
 }
 
 cudaError_t tc_x_q(const TcState&, const ExtractWave& w, const DevLayer* h_dev, DevStatus* d_status,
-                   cudaStream_t s) {
+                   bool skip_fused, cudaStream_t s) {
   int max_nb = 0;
   for (int i = w.l0; i < w.l1; ++i) max_nb = h_dev[i].NB > max_nb ? h_dev[i].NB : max_nb;
   const int stages = stages_for(max_nb);
   dim3 grid((w.max_m + 127) / 128, w.l1 - w.l0);
-  tc_x_q_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages);
+  tc_x_q_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages,
+                                                                   skip_fused ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -36,9 +36,17 @@ cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int
 
 cudaError_t tc_fill_omega(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,
                           uint64_t seed, cudaStream_t s);
+// skip_fused: leave out the layers that the fused power-step kernel serves (fz_C > 0)
 cudaError_t tc_xt_t(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,
-                    DevStatus* d_status, cudaStream_t s);
+                    DevStatus* d_status, bool skip_fused, cudaStream_t s);
 cudaError_t tc_x_q(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,
-                   DevStatus* d_status, cudaStream_t s);
+                   DevStatus* d_status, bool skip_fused, cudaStream_t s);
+
+// ---- fused power step (agzo_extract_fused.cu): Y = X^T (X Q) in one pass over X
+bool fused_eligible(const agzo_layer& a);
+int fused_cluster_size(const agzo_layer& a);
+cudaError_t fused_init();
+cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
+                                    int sm_count, cudaStream_t s);
 
 }  // namespace agzo

@@ -228,7 +228,15 @@ EXTRACT_CASES = [
     (333, 200, 16, 2, 32, True, 2),
     (640, 256, 24, 1, 32, True, 2),
     (512, 256, 64, 1, 0, True, 2),
-    (4096, 3072, 4, 3, 32, True, 2),     # several column chunks and slabs
+    (4096, 3072, 4, 3, 32, True, 2),     # several column chunks and slabs; fused power step on clusters of 6
+    (1024, 4096, 16, 2, 32, True, 2),    # fused power step, clusters of 8
+    (1536, 2048, 8, 3, 32, True, 2),     # clusters of 4
+    (900, 136, 3, 2, 8, True, 2),        # a single CTA per cluster, ragged token tile
+    # the same tensor-core products without the fused power step (two sweeps over X per step)
+    (2048, 1024, 8, 3, 32, True, 3),
+    (700, 520, 8, 3, 16, True, 3),
+    (333, 200, 16, 2, 32, True, 3),
+    (4096, 3072, 4, 3, 32, True, 3),
 ]
 
 
@@ -239,6 +247,7 @@ def _run_extract(X, r, K, seed, layer_id, path, x_bf16, pitch=None):
     layers = [B.make_layer(X=Xd, V=Vv, r=r, layer_id=layer_id)]
     with Ctx(layers) as ctx:
         B.agzo_set_option(ctx, "extract_path", path)
+        B.agzo_set_option(ctx, "extract_fused", 1 if path == 2 else 0)
         B.agzo_extract_subspace(ctx, layers, seed, K)
         st = B.agzo_poll(ctx)
     assert bool((Vd[0] == 7).all() and (Vd[-1] == 7).all() and (Vd[:, X.shape[1]:] == 7).all())
@@ -276,6 +285,28 @@ def test_extract_many_layers_in_waves():
         for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
             Vo = O.extract_subspace(X, r, 3, 3, i)
             assert projector_distance(to_host(devs[i][1]), Vo) <= 1e-3
+
+
+def test_extract_wave_mixes_fused_and_unfused_layers():
+    # d_in = 4608 and r = 24 are beyond the fused kernel's shapes; the others run fused on clusters of 2, 1 and 4
+    specs = [(640, 1024, 8), (512, 4608, 4), (700, 264, 16), (512, 512, 24), (768, 2048, 2)]
+    Xs = [WL.planted_activations(m, d, 16, seed=10 + i, bf16=True) for i, (m, d, r) in enumerate(specs)]
+    devs, layers = [], []
+    for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
+        Xd, _ = to_dev(X, True)
+        Vd = torch.zeros(r, d, device=DEV)
+        devs.append((Xd, Vd))
+        layers.append(B.make_layer(X=Xd, V=Vd, r=r, layer_id=i))
+    with Ctx(layers) as ctx:
+        B.agzo_set_option(ctx, "extract_path", 2)
+        B.agzo_set_option(ctx, "extract_fused", 1)
+        B.agzo_extract_subspace(ctx, layers, 5, 3)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
+        Vo = O.extract_subspace(X, r, 3, 5, i)
+        Vg = to_host(devs[i][1])
+        assert projector_distance(Vg, Vo) <= 1e-3
+        assert np.abs(Vg - Vo).max() <= 1e-3
 
 
 def test_extract_rank_deficient_panel_is_reported():
