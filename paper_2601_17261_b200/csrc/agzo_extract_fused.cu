@@ -15,10 +15,22 @@
 // As in the unfused kernels Q and T are fp32 quantities carried as hi + lo bf16 pairs in NB = 2 NP
 // operand columns (NP = r rounded up to 8), products exact, accumulation fp32.
 //
+// Status: correct (same parity tests as the two-sweep kernels) but not yet faster, so it is an
+// option ("extract_fused"), off by default.  Measured on B200 at d_in = 4096, r = 16, clusters of
+// 8: a tile's exchange takes about 4.4 us from the last phase-A MMA to the T operand being ready
+// (TMEM read 0.2, partial to shared memory + cluster-scope release arrive 1.0, slowest peer 0.6,
+// 16 remote loads per thread 1.5, second arrive + operand write 0.9).  The 176 KiB ring holds
+// 2.75 tiles of 64 KiB, each occupied for load + exchange + phase C (about 7 us), which caps a CTA
+// near 25 GB/s, 1.8 TB/s over the 120 CTAs that 15 resident clusters give -- below the 6.8 TB/s at
+// which the two-sweep kernels read X twice.  What would change this: a push-style reduce-scatter /
+// all-gather through st.async (one-way hops, an eighth of the traffic), or keeping the phase-C
+// operand out of shared memory (re-read of the tile from L2) so that the exchange latency no
+// longer ties up the ring.
+//
 // Roles in a CTA: warp 0 TMA producer (Q slice once per item, X slots of [64 tokens][128 columns]
 // through a ring), warp 1 MMA issuer (phase A of tile i+1 is issued before phase C of tile i so the
-// exchange of one tile overlaps the loads and phase A of the next), warps 2..5 epilogue (TMEM ->
-// exchange -> T operand; Y write-out).  Every wait is bounded; a wait that runs out sets the status
+// exchange of one tile overlaps the loads and phase A of the next), two groups of four epilogue warps
+// that take alternate tiles (TMEM -> exchange -> T operand; group 0 also writes Y out).  Every wait is bounded; a wait that runs out sets the status
 // word and the CTA leaves through the common exit (copies drained, cluster barrier, TMEM freed).
 #include <cuda.h>
 
@@ -31,7 +43,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kFzThreads = 192;
+constexpr int kFzThreads = 64 + 2 * 128;   // producer warp, MMA warp, two epilogue groups of four warps
 constexpr int kTT = 64;                    // tokens per tile
 constexpr int kSliceCols = 512;            // columns of X per CTA
 constexpr int kMBlocks = kSliceCols / 128; // M blocks of phase C
@@ -225,8 +237,11 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
     }
   } else {
     // ------------------------------------------------ epilogue warps
+    // Two groups of four warps take alternate tiles (group = parity of the tile counter), so the
+    // latency of one tile's exchange is hidden behind the other group's tile.
     const int q = warp & 3;                 // TMEM lanes 32q .. 32q+31
-    const int et = threadIdx.x - 64;        // 0..127 among the epilogue threads
+    const int grp = (warp - 2) >> 2;
+    const int et = threadIdx.x - 64 - 128 * grp;   // 0..127 inside the group
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     int te = 0, ic = 0;
     bool ok = true;
@@ -240,6 +255,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       const int hn = NP >> 1;               // values of a T row that one thread sums: NP/2
       for (int tile = 0; tile < it.ntiles && ok; ++tile, ++te) {
         const int p = te & 1, u2 = te >> 1;
+        if (p != grp) continue;
         ok = mbar_wait(&sh.tp_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -277,9 +293,8 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
               *reinterpret_cast<float4*>(dst + k4 * 4) =
                   make_float4(tsum[k4 * 4], tsum[k4 * 4 + 1], tsum[k4 * 4 + 2], tsum[k4 * 4 + 3]);
         }
-        named_bar_sync(1, 128);
-        if (et == 0)
-          for (int c = 0; c < C; ++c) mbar_arrive_cluster(mapa_shared(smem_u32(&sh.xch_full[p]), (uint32_t)c));
+        named_bar_sync(1 + grp, 128);
+        if (et < C) mbar_arrive_cluster(mapa_shared(smem_u32(&sh.xch_full[p]), (uint32_t)et));   // one peer per thread
         ok = mbar_wait_cluster(&sh.xch_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -289,18 +304,29 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] = 0.f;
         const uint32_t mine = smem_u32(xch + row * NP + kh);
-        for (int c = 0; c < C; ++c) {
-          const uint32_t ra = mapa_shared(mine, (uint32_t)c);
-          const float4 a = ld_cluster_f4(ra);
-          acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
-          if (hn == 8) {
-            const float4 b = ld_cluster_f4(ra + 16);
-            acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+        {
+          // all loads first (they are independent), then the sum in rank order
+          float4 va[8], vb[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            va[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            vb[c] = va[c];
+            if (c < C) {
+              const uint32_t ra = mapa_shared(mine, (uint32_t)c);
+              va[c] = ld_cluster_f4(ra);
+              if (hn == 8) vb[c] = ld_cluster_f4(ra + 16);
+            }
+          }
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            if (c < C) {
+              acc[0] += va[c].x; acc[1] += va[c].y; acc[2] += va[c].z; acc[3] += va[c].w;
+              acc[4] += vb[c].x; acc[5] += vb[c].y; acc[6] += vb[c].z; acc[7] += vb[c].w;
+            }
           }
         }
-        named_bar_sync(1, 128);              // every epilogue thread of this CTA has finished reading the peers
-        if (et == 0)
-          for (int c = 0; c < C; ++c) mbar_arrive_cluster(mapa_shared(smem_u32(&sh.xch_free[p]), (uint32_t)c));
+        named_bar_sync(1 + grp, 128);        // every thread of the group has finished reading the peers
+        if (et < C) mbar_arrive_cluster(mapa_shared(smem_u32(&sh.xch_free[p]), (uint32_t)et));
         // T operand of phase C: rows = hi parts 0..NP-1 then lo parts, 64 tokens (128 bytes) per row
         if (u2 > 0) {
           ok = mbar_wait(&sh.tt_empty[p], (u2 - 1) & 1);
@@ -323,6 +349,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         if (lane == 0) mbar_arrive(&sh.tt_full[p]);
       }
       if (!ok) break;
+      if (grp != 0) continue;
       // the item's partial Y: lanes = columns of the slice
       ok = mbar_wait(&sh.y_full, ic & 1);
       ok = __all_sync(0xffffffffu, ok);

@@ -194,14 +194,14 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
   const unsigned long long t0 = global_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < 64; ++i) {
       uint32_t ok;
       asm volatile(
           "{\n\t.reg .pred p;\n\t"
-          "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+          "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
           "selp.u32 %0, 1, 0, p;\n\t}"
           : "=r"(ok)
-          : "r"(smem_u32(bar)), "r"(parity), "r"(4000u)
+          : "r"(smem_u32(bar)), "r"(parity)
           : "memory");
       if (ok) return true;
     }
@@ -212,8 +212,7 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t remote_addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
                : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(remote_addr)
-               : "memory");
+               : "r"(remote_addr));
   return v;
 }
 // every thread of every CTA of the cluster
