@@ -97,7 +97,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- workload
-def build_layer_set(cfg: WL.LayerSetConfig, rank: int, device, seed: int = 1000):
+def build_layer_set(cfg: WL.LayerSetConfig, rank: int, device, seed: int = 1000, alias_inputs: bool = False):
     """Resident tensors of one layer set: bf16 W and X per layer (torch device generators,
     same recipe as the host generators the parity tests use), fp32 V."""
     from paper_2601_17261_b200 import binding as B
@@ -106,16 +106,22 @@ def build_layer_set(cfg: WL.LayerSetConfig, rank: int, device, seed: int = 1000)
     Ws, Xs, Vs, layers = [], [], [], []
     for i, (name, d_in, d_out) in enumerate(cfg.layers()):
         W = WL.device_weights(d_out, d_in, cfg.w_std, gen, device)
-        X = WL.device_planted_activations(cfg.m, d_in, cfg.planted_rank, gen, device)
+        kind = name.split(".")[-1]
+        if alias_inputs and kind in ("k", "v", "up"):
+            X = Xs[-1]          # k, v read q's input; up reads gate's: one buffer, as in a transformer block
+        else:
+            X = WL.device_planted_activations(cfg.m, d_in, cfg.planted_rank, gen, device)
         V = torch.zeros(rank, d_in, dtype=torch.float32, device=device)
         Ws.append(W); Xs.append(X); Vs.append(V)
         layers.append(B.make_layer(W=W, X=X, V=V, r=rank, layer_id=i))
     return Ws, Xs, Vs, layers
 
 
-def algorithmic_work(cfg: WL.LayerSetConfig, rank: int):
+def algorithmic_work(cfg: WL.LayerSetConfig, rank: int, alias_inputs: bool = False):
     n_w = cfg.n_params()
     x_elems = cfg.x_elems()
+    if alias_inputs:   # q/k/v and gate/up read one buffer each: distinct activation bytes only
+        x_elems = cfg.n_blocks * sum(cfg.m * di for (nm, di, _) in cfg.block if nm not in ("k", "v", "up"))
     rmw_bytes_pass = 4 * n_w + sum(4 * rank * di for (_, di, _) in cfg.layers())
     extract_bytes = (K_POWER + 1) * 2 * x_elems          # X read once per product pair (fused)
     extract_bytes_unfused = (2 * K_POWER + 1) * 2 * x_elems
@@ -200,6 +206,9 @@ def main():
     ap.add_argument("--wave-mb", type=int, default=-1)
     ap.add_argument("--extract-streams", type=int, default=2)
     ap.add_argument("--extract-fused", type=int, default=0)
+    ap.add_argument("--alias-inputs", action="store_true",
+                    help="q/k/v and gate/up of a block read one activation buffer each (as in a real block)")
+    ap.add_argument("--share-inputs", type=int, default=1)
     ap.add_argument("--rmw-path", type=int, default=0)
     ap.add_argument("--rmw-slots", type=int, default=0)
     ap.add_argument("--rmw-inflight", type=int, default=0)
@@ -233,7 +242,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     B.lib()   # fails loudly when the CUDA library is missing
 
-    Ws, Xs, Vs, layers = build_layer_set(cfg, r, dev)
+    Ws, Xs, Vs, layers = build_layer_set(cfg, r, dev, alias_inputs=args.alias_inputs)
     arr = B.layer_array(layers)
     # a larger wave than the default needs more scratch than agzo_workspace_bytes reports
     ctx = B.agzo_create(layers, local, extra_bytes=(12 << 30) if args.wave_mb > 4096 else 0)
@@ -241,12 +250,13 @@ def main():
     B.agzo_set_option(ctx, "rmw_path", args.rmw_path)
     B.agzo_set_option(ctx, "extract_streams", args.extract_streams)
     B.agzo_set_option(ctx, "extract_fused", args.extract_fused)
+    B.agzo_set_option(ctx, "share_inputs", args.share_inputs)
     B.agzo_set_option(ctx, "rmw_tc_slots", args.rmw_slots)
     B.agzo_set_option(ctx, "rmw_tc_inflight", args.rmw_inflight)
     B.agzo_set_option(ctx, "rmw_tc_panels", args.rmw_panels)
     if args.wave_mb >= 0:
         B.agzo_set_option(ctx, "wave_bytes", args.wave_mb << 20)
-    work = algorithmic_work(cfg, r)
+    work = algorithmic_work(cfg, r, args.alias_inputs)
     losses = torch.tensor([1.0, 0.999], dtype=torch.float64, device=dev)
     ghat = torch.zeros(1, device=dev)
     stream = torch.cuda.current_stream()
@@ -353,7 +363,9 @@ def main():
                                    f"m={cfg.m} tokens, r={r}, K={K_POWER}, eps={EPS}, two-point",
                        "l2": "inputs larger than L2 (weights %.1f GB + activations %.1f GB per step)"
                              % (work["w_bytes"] / 1e9, work["x_bytes"] / 1e9),
-                       "replicas": world, "device_status": B.status_string(status)},
+                       "replicas": world, "device_status": B.status_string(status),
+                       "inputs": ("q/k/v and gate/up share one activation buffer per block" if args.alias_inputs
+                                  else "one activation buffer per layer")},
             "phases_ms": {"extract": ms_extract, "perturb": ms_perturb, "restore_update": ms_update},
             "rmw": {"GBps_perturb": work["rmw_bytes_per_pass"] / ms_perturb / 1e6,
                     "GBps_restore_update": work["rmw_bytes_per_pass"] / ms_update / 1e6,

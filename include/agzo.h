@@ -127,6 +127,9 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * for every layer that allows it; tuning knobs of that kernel, 0 = chosen by rank:
  * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),
  * "rmw_tc_panels" (column panels per work item, 1 or 2);
+ * "share_inputs" 1 (default) = consecutive layers whose X is the same buffer (same pointer, pitch,
+ * m, d_in: q/k/v or gate/up of a transformer block) are served by one sweep over X per product,
+ * with identical results; 0 = every layer sweeps its X itself;
  * "extract_fused" 1 = layers with r <= 16 and d_in <= 4096 on the tensor-core path run each
  * power step in the fused kernel that reads X once (thread-block clusters); 0 = off;
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;

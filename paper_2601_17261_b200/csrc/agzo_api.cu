@@ -45,6 +45,7 @@ struct PlanOpts {
   int rmw_tc_panels;     // column panels per work item of the tensor-core pass (1 or 2)
   bool tc_available;
   bool extract_fused;    // power steps of eligible layers run in the fused single-pass kernel
+  bool share_inputs;     // consecutive layers with the same X are served by one sweep
   int extract_regions;   // 1: waves run one after another; 2: alternate waves use two scratch regions
                          // and two helper streams, so one wave's small kernels overlap the other's sweeps
 };
@@ -67,6 +68,7 @@ struct agzo_ctx {
   int64_t wave_bytes;
   int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
   int extract_fused;       // 1: fused power-step kernel where a layer's shape allows it
+  int share_inputs;        // 1: consecutive layers with the same X share the sweeps over it
   cudaStream_t aux[2];     // helper streams of extraction, forked from and joined to the caller's stream
   cudaEvent_t fork_ev, join_ev[2];
   // descriptors last uploaded
@@ -157,6 +159,9 @@ agzo_status validate(const agzo_layer* L, int n, int need) {
 }
 
 bool has_x(const agzo_layer& a) { return a.X != nullptr && a.m >= 1; }
+bool same_input(const agzo_layer& a, const agzo_layer& b) {
+  return a.X == b.X && a.ldx == b.ldx && a.m == b.m && a.d_in == b.d_in && a.x_dtype == b.x_dtype;
+}
 
 // Token slabs of the X^T T product.  CUDA-core kernels: 32 slabs at most.  Tensor-core
 // kernels: slabs of 2048 tokens (32 pipeline steps per CTA) when the layer has that many; a
@@ -176,7 +181,7 @@ void slab_shape(const agzo_layer& a, bool tc, int* slabs, int* slab_rows) {
 }
 
 // scratch bytes one layer needs for extraction (0 when it has no X)
-size_t layer_scratch(const agzo_layer& a, bool tc) {
+size_t layer_scratch(const agzo_layer& a, bool tc, bool with_panels = true) {
   if (!has_x(a)) return 0;
   int slabs, slab_rows;
   slab_shape(a, tc, &slabs, &slab_rows);
@@ -188,7 +193,7 @@ size_t layer_scratch(const agzo_layer& a, bool tc) {
   b += align_up(r * d * 4);                 // Y
   b += align_up(gch * r * r * 8);           // Gpart
   b += align_up(r * r * 8);                 // M
-  if (tc) b += tc_layer_scratch(a);
+  if (tc && with_panels) b += tc_layer_scratch(a);
   return b;
 }
 
@@ -283,35 +288,66 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
     while (j < n && has_x(L[j])) {
       const bool tc = extract_path != 1 && tc_available && tc_eligible(L[j]);
       if (tc != wave_tc) break;      // a wave runs on one kind of kernel
-      const size_t need = layer_scratch(L[j], tc);
+      // a unit is one layer, or a run of consecutive layers that read the same X (one sweep serves all)
+      int glen = 1, rows = tc ? tc_operand_rows(L[j].r) : 0;
+      if (tc && opts.share_inputs && !opts.extract_fused) {
+        while (j + glen < n && has_x(L[j + glen]) && same_input(L[j], L[j + glen]) && tc_eligible(L[j + glen]) &&
+               rows + tc_operand_rows(L[j + glen].r) <= 256) {
+          rows += tc_operand_rows(L[j + glen].r);
+          ++glen;
+        }
+      }
+      auto unit_need = [&](int len, int nrows) {
+        size_t b = 0;
+        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, false);
+        if (tc) b += tc_panel_bytes(L[j], nrows);
+        return b;
+      };
+      size_t need = unit_need(glen, rows);
       const int64_t xb = (int64_t)L[j].m * L[j].d_in * (L[j].x_dtype == AGZO_BF16 ? 2 : 4);
       if (j > i && (used + need > scratch_cap || xbytes + xb > wave_bytes)) break;
+      if (used + need > scratch_cap && glen > 1) {   // the group alone does not fit: fall back to single layers
+        glen = 1;
+        rows = tc_operand_rows(L[j].r);
+        need = unit_need(glen, rows);
+      }
       if (used + need > scratch_cap) return AGZO_ERR_WORKSPACE;
       // carve
       if (ws) {
         char* p = ws + base + (size_t)region * scratch_cap + used;
-        DevLayer& D = plan->dev[j];
-        const agzo_layer& a = L[j];
-        int slabs, slab_rows;
-        slab_shape(a, tc, &slabs, &slab_rows);
-        const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
-        const size_t gch = (d + 127) / 128;
-        D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
-        D.T = reinterpret_cast<float*>(p);      p += align_up(m * r * 4);
-        D.Ypart = reinterpret_cast<float*>(p);  p += align_up((size_t)slabs * r * d * 4);
-        D.Y = reinterpret_cast<float*>(p);      p += align_up(r * d * 4);
-        D.Gpart = reinterpret_cast<double*>(p); p += align_up(gch * r * r * 8);
-        D.M = reinterpret_cast<double*>(p);     p += align_up(r * r * 8);
+        for (int g = 0; g < glen; ++g) {
+          DevLayer& D = plan->dev[j + g];
+          const agzo_layer& a = L[j + g];
+          int slabs, slab_rows;
+          slab_shape(a, tc, &slabs, &slab_rows);
+          const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
+          const size_t gch = (d + 127) / 128;
+          D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
+          D.T = reinterpret_cast<float*>(p);      p += align_up(m * r * 4);
+          D.Ypart = reinterpret_cast<float*>(p);  p += align_up((size_t)slabs * r * d * 4);
+          D.Y = reinterpret_cast<float*>(p);      p += align_up(r * d * 4);
+          D.Gpart = reinterpret_cast<double*>(p); p += align_up(gch * r * r * 8);
+          D.M = reinterpret_cast<double*>(p);     p += align_up(r * r * 8);
+        }
         if (tc) {
-          tc_carve(a, &D, p);
-          D.tmaps = ws + maps_offset(n) + (size_t)j * kMapBytes;
-          // the power steps of this layer run fused (X read once per step) where its shape allows
-          D.fz_C = (opts.extract_fused && extract_path != 3 && fused_eligible(a)) ? fused_cluster_size(a) : 0;
+          int row0 = 0;
+          for (int g = 0; g < glen; ++g) {
+            DevLayer& D = plan->dev[j + g];
+            const agzo_layer& a = L[j + g];
+            tc_set_panels(a, &D, p, rows, row0);
+            row0 += tc_operand_rows(a.r);
+            D.grp_role = glen == 1 ? 0 : (g == 0 ? 1 : 2);
+            D.grp_n = g == 0 ? glen : 0;
+            D.grp_NB = g == 0 ? rows : 0;
+            D.tmaps = ws + maps_offset(n) + (size_t)(j + g) * kMapBytes;
+            // the power steps of this layer run fused (X read once per step) where its shape allows
+            D.fz_C = (opts.extract_fused && extract_path != 3 && fused_eligible(a)) ? fused_cluster_size(a) : 0;
+          }
         }
       }
       used += need;
       xbytes += xb;
-      ++j;
+      j += glen;
     }
     if (used > max_wave_scratch) max_wave_scratch = used;
     plan->wave_end.push_back(j);
@@ -341,7 +377,7 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
   PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels,
-                c->tc.available, c->extract_fused != 0, c->extract_streams};
+                c->tc.available, c->extract_fused != 0, c->share_inputs != 0, c->extract_streams};
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
     opts.extract_regions = 1;
@@ -369,7 +405,8 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
     std::memcpy(hs + lb + (size_t)(n + 1) * sizeof(int), plan.item_start.data(), (size_t)(n + 1) * sizeof(int));
     char* hmaps = hs + lb + prefix_bytes(n);
     for (int i = 0; i < n; ++i) {
-      if (plan.dev[i].Qb && !tc_encode_maps(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes))
+      if (plan.dev[i].Qb && plan.dev[i].grp_role != 2 &&
+          !tc_encode_maps(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes))
         return AGZO_ERR_UNSUPPORTED;
       if (plan.dev[i].wmap && !rmw_tc_encode_map(c->tc, plan.dev[i], hmaps + (size_t)i * kMapBytes + 384))
         return AGZO_ERR_UNSUPPORTED;
@@ -444,9 +481,9 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true, false, 2}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true, false, false, 2}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false, false, 2}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false, false, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -478,6 +515,7 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->wave_bytes = kDefaultWaveBytes;
   c->extract_streams = 2;
   c->extract_fused = 0;
+  c->share_inputs = 1;
   c->aux[0] = c->aux[1] = nullptr;
   c->fork_ev = c->join_ev[0] = c->join_ev[1] = nullptr;
   c->cached_valid = false;
@@ -553,6 +591,9 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
     if (value < 0 || value > 64) return AGZO_ERR_INVALID_ARG;
     ctx->rmw_tc_slots = (int)value;
     return AGZO_OK;
+  } else if (std::strcmp(name, "share_inputs") == 0) {
+    if (value < 0 || value > 1) return AGZO_ERR_INVALID_ARG;
+    ctx->share_inputs = (int)value;
   } else if (std::strcmp(name, "extract_fused") == 0) {
     if (value < 0 || value > 1) return AGZO_ERR_INVALID_ARG;
     ctx->extract_fused = (int)value;

@@ -39,6 +39,13 @@ struct alignas(16) DevLayer {
   long long m_pad;       // row pitch of Tb in elements (m rounded up to 8)
   int NB, NP;
   int fz_C;              // cluster size of the fused power-step kernel for this layer, 0 = unfused kernels
+  // Consecutive layers that read the same X (q/k/v, gate/up of a transformer block) form a group:
+  // their operand panels are adjacent rows of one matrix, the leader's CTAs run both products
+  // for all members with N = grp_NB columns, and X is read once per product for the group.
+  int grp_role;          // 0 single layer, 1 group leader, 2 member (served by its leader)
+  int grp_n;             // leader: number of layers in the group (itself included)
+  int grp_NB;            // leader: operand rows of the whole group
+  int grp_off;           // first operand row of this layer inside the group's panels
   // tensor-core in-place pass (bf16 W): this layer's work items are
   // [rtc_item0, rtc_item0 + rtc_panels * rtc_chunks); item = (row chunk, group of column panels)
   const void* wmap;      // 128-byte TMA descriptor of W, box = 64 columns x 128 rows; null = CUDA-core pass

@@ -58,11 +58,12 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
                                                             DevStatus* status, int stages, int skip_fused) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const int t0 = blockIdx.x * 128;
-  if (t0 >= L.m || (skip_fused && L.fz_C)) return;
+  if (t0 >= L.m || (skip_fused && L.fz_C) || L.grp_role == 2) return;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ TcShared sh;
-  const int NB = L.NB, NP = L.NP;
+  const int NB = L.grp_role == 1 ? L.grp_NB : L.NB;   // operand rows: the whole group's for a leader
+  const int nmem = L.grp_role == 1 ? L.grp_n : 1;
   const int a_bytes = 2 * kTileBytes;                 // [128 tokens][64 d]
   const int b_bytes = NB * kBoxK * 2;                 // [NB][64 d]
   const int stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023);
@@ -127,20 +128,24 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
     tc_fence_after();
     if (!ok) sh.failed = 1;
     const int t = t0 + q * 32 + lane;
-    __nv_bfloat16* Tt = L.Tb;
-    const long long mp = L.m_pad;
     if (ok) {
-      for (int k0 = 0; k0 < NP; k0 += 8) {
-        float hi[8], lo[8];
-        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)k0, hi);
-        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(NP + k0), lo);
-        if (t < L.m) {
+      for (int mi = 0; mi < nmem; ++mi) {               // the layers this CTA serves
+        const DevLayer& M = layers[l0 + blockIdx.y + mi];
+        const int NP = M.NP, off = L.grp_role == 1 ? M.grp_off : 0;
+        __nv_bfloat16* Tt = M.Tb;
+        const long long mp = M.m_pad;
+        for (int k0 = 0; k0 < NP; k0 += 8) {
+          float hi[8], lo[8];
+          tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(off + k0), hi);
+          tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(off + NP + k0), lo);
+          if (t < L.m) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            __nv_bfloat16 h, l;
-            split_bf16(hi[j] + lo[j], &h, &l);
-            Tt[(long long)(k0 + j) * mp + t] = h;
-            Tt[(long long)(NP + k0 + j) * mp + t] = l;
+            for (int j = 0; j < 8; ++j) {
+              __nv_bfloat16 h, l;
+              split_bf16(hi[j] + lo[j], &h, &l);
+              Tt[(long long)(k0 + j) * mp + t] = h;
+              Tt[(long long)(NP + k0 + j) * mp + t] = l;
+            }
           }
         }
       }
@@ -159,11 +164,12 @@ __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __r
   const DevLayer& L = layers[l0 + blockIdx.z];
   const int d0 = blockIdx.x * 128;
   const int slab = blockIdx.y;
-  if (d0 >= L.d_in || slab >= L.slabs || (skip_fused && L.fz_C)) return;
+  if (d0 >= L.d_in || slab >= L.slabs || (skip_fused && L.fz_C) || L.grp_role == 2) return;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ TcShared sh;
-  const int NB = L.NB, NP = L.NP;
+  const int NB = L.grp_role == 1 ? L.grp_NB : L.NB;
+  const int nmem = L.grp_role == 1 ? L.grp_n : 1;
   const int a_bytes = 2 * kTileBytes;                 // two [64 tokens][64 d] boxes: d0.., d0+64..
   const int b_bytes = NB * kBoxK * 2;                 // [NB][64 tokens]
   const int stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023);
@@ -231,17 +237,20 @@ __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __r
     tc_fence_after();
     if (!ok) sh.failed = 1;
     const int d = d0 + q * 32 + lane;
-    const int r = L.r;
     if (ok) {
-      float* out = L.Ypart + (long long)slab * r * L.d_in + d;
-      for (int k0 = 0; k0 < NP; k0 += 8) {
-        float hi[8], lo[8];
-        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)k0, hi);
-        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(NP + k0), lo);
-        if (d < L.d_in) {
+      for (int mi = 0; mi < nmem; ++mi) {               // the layers this CTA serves (same slabs: same m)
+        const DevLayer& M = layers[l0 + blockIdx.z + mi];
+        const int r = M.r, NP = M.NP, off = L.grp_role == 1 ? M.grp_off : 0;
+        float* out = M.Ypart + (long long)slab * r * L.d_in + d;
+        for (int k0 = 0; k0 < NP; k0 += 8) {
+          float hi[8], lo[8];
+          tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(off + k0), hi);
+          tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(off + NP + k0), lo);
+          if (d < L.d_in) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (k0 + j < r) out[(long long)(k0 + j) * L.d_in] = hi[j] + lo[j];
+            for (int j = 0; j < 8; ++j)
+              if (k0 + j < r) out[(long long)(k0 + j) * L.d_in] = hi[j] + lo[j];
+          }
         }
       }
     }
@@ -365,18 +374,23 @@ bool tc_eligible(const agzo_layer& a) {
          a.d_in % 8 == 0 && a.d_in >= 128 && a.m >= 256 && a.r >= 1 && a.r <= AGZO_MAX_RANK;
 }
 
-size_t tc_layer_scratch(const agzo_layer& a) {
-  const size_t NB = 2 * (size_t)np_of(a.r);
-  return up256(NB * (size_t)a.d_in * 2) + up256(NB * (size_t)mpad_of(a.m) * 2);
+int tc_operand_rows(int r) { return 2 * np_of(r); }
+
+size_t tc_panel_bytes(const agzo_layer& a, int rows) {
+  return up256((size_t)rows * (size_t)a.d_in * 2) + up256((size_t)rows * (size_t)mpad_of(a.m) * 2);
 }
 
-void tc_carve(const agzo_layer& a, DevLayer* D, char* p) {
+size_t tc_layer_scratch(const agzo_layer& a) { return tc_panel_bytes(a, tc_operand_rows(a.r)); }
+
+void tc_set_panels(const agzo_layer& a, DevLayer* D, char* p, int rows, int row0) {
   D->NP = np_of(a.r);
   D->NB = 2 * D->NP;
   D->m_pad = mpad_of(a.m);
-  D->Qb = reinterpret_cast<__nv_bfloat16*>(p);
-  p += up256((size_t)D->NB * a.d_in * 2);
-  D->Tb = reinterpret_cast<__nv_bfloat16*>(p);
+  __nv_bfloat16* qb = reinterpret_cast<__nv_bfloat16*>(p);
+  __nv_bfloat16* tb = reinterpret_cast<__nv_bfloat16*>(p + up256((size_t)rows * (size_t)a.d_in * 2));
+  D->Qb = qb + (size_t)row0 * a.d_in;
+  D->Tb = tb + (size_t)row0 * D->m_pad;
+  D->grp_off = row0;
 }
 
 bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps) {
@@ -384,13 +398,13 @@ bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps) {
   uint8_t* out = static_cast<uint8_t*>(host_maps);
   // X [m][ldx]: inner = d_in, outer = m; one box = 64 columns x 64 tokens
   if (!encode_2d(st.encode_fn, out, D.X, (uint64_t)D.d_in, (uint64_t)D.m, (uint64_t)D.ldx * 2, 64, 64)) return false;
-  // Qb [NB][d_in]: box = 64 columns x NB rows
-  if (!encode_2d(st.encode_fn, out + 128, D.Qb, (uint64_t)D.d_in, (uint64_t)D.NB, (uint64_t)D.d_in * 2, 64,
-                 (uint32_t)D.NB))
+  // a group leader's descriptors cover the operand rows of the whole group
+  const uint32_t nb = D.grp_role == 1 ? (uint32_t)D.grp_NB : (uint32_t)D.NB;
+  // Qb [nb][d_in]: box = 64 columns x nb rows
+  if (!encode_2d(st.encode_fn, out + 128, D.Qb, (uint64_t)D.d_in, (uint64_t)nb, (uint64_t)D.d_in * 2, 64, nb))
     return false;
-  // Tt [NB][m_pad]: inner extent is the true m so that the padding is read as zero
-  if (!encode_2d(st.encode_fn, out + 256, D.Tb, (uint64_t)D.m, (uint64_t)D.NB, (uint64_t)D.m_pad * 2, 64,
-                 (uint32_t)D.NB))
+  // Tt [nb][m_pad]: inner extent is the true m so that the padding is read as zero
+  if (!encode_2d(st.encode_fn, out + 256, D.Tb, (uint64_t)D.m, (uint64_t)nb, (uint64_t)D.m_pad * 2, 64, nb))
     return false;
   return true;
 }
@@ -407,7 +421,10 @@ cudaError_t tc_fill_omega(const TcState&, const ExtractWave& w, const DevLayer*,
 cudaError_t tc_xt_t(const TcState&, const ExtractWave& w, const DevLayer* h_dev, DevStatus* d_status,
                     bool skip_fused, cudaStream_t s) {
   int max_nb = 0;
-  for (int i = w.l0; i < w.l1; ++i) max_nb = h_dev[i].NB > max_nb ? h_dev[i].NB : max_nb;
+  for (int i = w.l0; i < w.l1; ++i) {
+    const int nb = h_dev[i].grp_role == 1 ? h_dev[i].grp_NB : h_dev[i].NB;
+    max_nb = nb > max_nb ? nb : max_nb;
+  }
   const int stages = stages_for(max_nb);
   dim3 grid((w.max_din + 127) / 128, w.max_slabs, w.l1 - w.l0);
   tc_xt_t_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages,
@@ -418,7 +435,10 @@ cudaError_t tc_xt_t(const TcState&, const ExtractWave& w, const DevLayer* h_dev,
 cudaError_t tc_x_q(const TcState&, const ExtractWave& w, const DevLayer* h_dev, DevStatus* d_status,
                    bool skip_fused, cudaStream_t s) {
   int max_nb = 0;
-  for (int i = w.l0; i < w.l1; ++i) max_nb = h_dev[i].NB > max_nb ? h_dev[i].NB : max_nb;
+  for (int i = w.l0; i < w.l1; ++i) {
+    const int nb = h_dev[i].grp_role == 1 ? h_dev[i].grp_NB : h_dev[i].NB;
+    max_nb = nb > max_nb ? nb : max_nb;
+  }
   const int stages = stages_for(max_nb);
   dim3 grid((w.max_m + 127) / 128, w.l1 - w.l0);
   tc_x_q_kernel<<<grid, kTcThreads, smem_for(max_nb, stages), s>>>(w.d_layers, w.l0, d_status, stages,

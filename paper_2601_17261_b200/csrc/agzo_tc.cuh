@@ -15,8 +15,11 @@ cudaError_t tc_init(TcState* st, int device);
 // true when the layer's activations can go through the tensor-core kernels
 bool tc_eligible(const agzo_layer& a);
 size_t tc_layer_scratch(const agzo_layer& a);
-// assigns Qb / Tb / NB / NP of D from scratch starting at p (after the common slices)
-void tc_carve(const agzo_layer& a, DevLayer* D, char* p);
+// operand rows of one layer (hi + lo parts of r rounded up to 8) and bytes of panels with `rows` rows
+int tc_operand_rows(int r);
+size_t tc_panel_bytes(const agzo_layer& a, int rows);   // Qb [rows][d_in] + Tb [rows][m_pad], each 256-byte padded
+// points D at rows [row0, row0 + its operand rows) of panels that start at p and have `rows` rows
+void tc_set_panels(const agzo_layer& a, DevLayer* D, char* p, int rows, int row0);
 
 // writes the layer's TMA descriptors (512 bytes) into host memory; false when encoding fails
 bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps);

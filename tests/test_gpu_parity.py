@@ -309,6 +309,35 @@ def test_extract_wave_mixes_fused_and_unfused_layers():
         assert np.abs(Vg - Vo).max() <= 1e-3
 
 
+def test_layers_that_share_their_input_are_served_by_one_sweep():
+    # q/k/v-like and gate/up-like groups on shared X buffers, a layer of its own in between
+    shapes = [(1024, 512), (640, 264), (900, 1024)]
+    Xh = [WL.planted_activations(m, d, 16, seed=20 + i, bf16=True) for i, (m, d) in enumerate(shapes)]
+    Xd = [to_dev(x, True, pitch=x.shape[1] + 8 if x.shape[1] % 16 else None)[0] for x in Xh]
+    plan = [(0, 8), (0, 4), (0, 16), (1, 5), (2, 8), (2, 8)]      # (which X, r)
+    results = {}
+    for share in (1, 0):
+        Vs, layers = [], []
+        for i, (xi, r) in enumerate(plan):
+            V = torch.zeros(r, Xh[xi].shape[1], device=DEV)
+            Vs.append(V)
+            layers.append(B.make_layer(X=Xd[xi], V=V, r=r, layer_id=40 + i))
+        with Ctx(layers) as ctx:
+            B.agzo_set_option(ctx, "extract_path", 3)
+            B.agzo_set_option(ctx, "share_inputs", share)
+            B.agzo_extract_subspace(ctx, layers, 9, 3)
+            assert B.agzo_poll(ctx) == B.AGZO_OK
+        results[share] = [to_host(V) for V in Vs]
+    for i, (xi, r) in enumerate(plan):
+        Vo = O.extract_subspace(Xh[xi], r, 3, 9, 40 + i)
+        Vg = results[1][i]
+        assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
+        assert projector_distance(Vg, Vo) <= 1e-3
+        assert np.abs(Vg - Vo).max() <= 1e-3
+        # grouping changes which CTA computes a column, not what is computed
+        assert np.abs(Vg - results[0][i]).max() <= 1e-6
+
+
 def test_extract_rank_deficient_panel_is_reported():
     rng = np.random.default_rng(0)
     m, d_in, r = 256, 128, 4
