@@ -5,8 +5,9 @@
 // thread-block cluster of C CTAs shares a tile of 64 tokens; CTA c keeps its 512-column slice of
 // the tile in shared memory while
 //   phase A   its slice's contribution to T (64 x NB, tcgen05.mma M = 64, K = 512) goes to TMEM,
-//   exchange  the C partial sums are added up through distributed shared memory (every CTA reads
-//             all C partials in rank order, so all of them hold the same T),
+//   exchange  the C partial sums are added up through distributed shared memory in two one-way
+//             hops (st.async): each row of the tile is summed in rank order by the CTA that owns
+//             it, and the sum is sent to every CTA, so all of them hold the same T,
 //   phase C   Y_slice (512 x NB, kept in TMEM across all tiles of the work item) += X_slice^T T
 //             (tcgen05.mma M = 128, the resident X boxes read as an MN-major operand).
 // X therefore crosses HBM once per power step.  A work item is (layer, token slab); the slab's
@@ -15,17 +16,17 @@
 // As in the unfused kernels Q and T are fp32 quantities carried as hi + lo bf16 pairs in NB = 2 NP
 // operand columns (NP = r rounded up to 8), products exact, accumulation fp32.
 //
-// Status: correct (same parity tests as the two-sweep kernels) but not yet faster, so it is an
-// option ("extract_fused"), off by default.  Measured on B200 at d_in = 4096, r = 16, clusters of
-// 8: a tile's exchange takes about 4.4 us from the last phase-A MMA to the T operand being ready
-// (TMEM read 0.2, partial to shared memory + cluster-scope release arrive 1.0, slowest peer 0.6,
-// 16 remote loads per thread 1.5, second arrive + operand write 0.9).  The 176 KiB ring holds
-// 2.75 tiles of 64 KiB, each occupied for load + exchange + phase C (about 7 us), which caps a CTA
-// near 25 GB/s, 1.8 TB/s over the 120 CTAs that 15 resident clusters give -- below the 6.8 TB/s at
-// which the two-sweep kernels read X twice.  What would change this: a push-style reduce-scatter /
-// all-gather through st.async (one-way hops, an eighth of the traffic), or keeping the phase-C
-// operand out of shared memory (re-read of the tile from L2) so that the exchange latency no
-// longer ties up the ring.
+// Status: correct (same parity tests as the two-sweep kernels) but not faster, so it is an option
+// ("extract_fused"), off by default.  Measured on B200 at d_in = 4096, r = 16, clusters of 8
+// (timestamps taken inside the kernel): the exchange takes 1.35 us from the last phase-A MMA to
+// the T operand being ready (it took 4.4 us with remote loads and cluster-scope release arrives),
+// but a tile still takes 3.5 us, because its 32 + 16 tcgen05.mma instructions (M = 64 or 128,
+// N = 32, K = 16) cost about 65 to 80 ns each whatever their size -- neither fewer instructions
+// in the issuing thread nor independent accumulators changed that.  64 KiB per 3.5 us is 19 GB/s
+// per CTA, 2.3 TB/s over the 120 CTAs of 15 resident clusters, against the 6.8 TB/s at which the
+// two-sweep kernels read X twice (they need one such instruction per 4 KiB of X and run two CTAs
+// per SM).  A fused step needs a product shape with more work per instruction (the 256-wide N
+// side on X, tiles of 128 or more tokens) before it can win.
 //
 // Roles in a CTA: warp 0 TMA producer (Q slice once per item, X slots of [64 tokens][128 columns]
 // through a ring), warp 1 MMA issuer (phase A of tile i+1 is issued before phase C of tile i so the
@@ -50,6 +51,7 @@ constexpr int kMBlocks = kSliceCols / 128; // M blocks of phase C
 constexpr int kSlotBytes = 16 * 1024;      // [64 tokens][128 columns] as two boxes of 64 columns
 constexpr int kBoxBytes = 8 * 1024;
 constexpr int kMaxRing = 12;
+constexpr int kRsFloats = 72 * 16;         // C * ceil(64 / C) <= 72 rows of up to 16 floats
 constexpr uint32_t kFzTmemCols = 256;
 
 struct FzShared {
@@ -57,7 +59,7 @@ struct FzShared {
   uint64_t qb_full, qb_empty;
   uint64_t tp_full[2], tp_empty[2];     // T partial in TMEM
   uint64_t tt_full[2], tt_empty[2];     // T operand in shared memory
-  uint64_t xch_full[2], xch_free[2];    // exchange buffers: all partials written / all peers done reading mine
+  uint64_t rs_full[2], ag_full[2];      // exchange: contributions to my rows have landed / the summed T has landed
   uint64_t y_full, y_free;
   uint32_t tmem_base;
   int failed;
@@ -99,12 +101,14 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
   const int rank = (int)cluster_ctarank();
   const int cluster = (int)cluster_id_x(), nclusters = (int)cluster_count_x();
   const int col0 = rank * kSliceCols;
-  // shared-memory carve-up: X ring | Q slice (8 boxes of [NB][64]) | T operand x2 | exchange x2
+  // shared-memory carve-up: X ring | Q slice (8 boxes of [NB][64]) | T operand x2 | exchange buffers x2
   uint8_t* sX = base;
   uint8_t* sQ = sX + (size_t)ring * kSlotBytes;
   // NB is a per-layer quantity; the regions are sized for NB = 32
   uint8_t* sTt = sQ + 8 * 32 * 128;
-  float* sXch = reinterpret_cast<float*>(sTt + 2 * 32 * 128);   // 2 x [64][16] floats
+  float* sRs = reinterpret_cast<float*>(sTt + 2 * 32 * 128);    // 2 x [C][rows_per][NP] floats
+  float* sAg = sRs + 2 * kRsFloats;                               // 2 x [64][16] floats
+  const int rows_per = (kTT + C - 1) / C;                         // token rows of a tile that one CTA sums
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < ring; ++s) { mbar_init(&sh.x_full[s], 1); mbar_init(&sh.x_empty[s], 1); }
@@ -112,7 +116,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
     for (int p = 0; p < 2; ++p) {
       mbar_init(&sh.tp_full[p], 1); mbar_init(&sh.tp_empty[p], 4);
       mbar_init(&sh.tt_full[p], 4); mbar_init(&sh.tt_empty[p], 1);
-      mbar_init(&sh.xch_full[p], C); mbar_init(&sh.xch_free[p], C);
+      mbar_init(&sh.rs_full[p], 1); mbar_init(&sh.ag_full[p], 1);
     }
     mbar_init(&sh.y_full, 1); mbar_init(&sh.y_free, 4);
     sh.failed = 0;
@@ -278,55 +282,58 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.tp_empty[p]);
-        // my partial -> my exchange buffer, once every peer has finished with its previous content
-        if (u2 > 0) {
-          ok = mbar_wait_cluster(&sh.xch_free[p], (u2 - 1) & 1);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
+        // Exchange, two one-way hops through st.async (data and its completion travel together):
+        //   reduce-scatter  row R of my partial goes to the CTA that owns R (rows_per rows each);
+        //   all-gather      the owner adds the C contributions in rank order and sends the sum to everyone.
+        // No buffer needs a "free" signal: a peer can only send tile i+2's data after it has received
+        // my tile-i sums, which I send after consuming the tile-i contributions.
+        float* rs = sRs + p * kRsFloats;          // [C sources][rows_per][NP]
+        float* ag = sAg + p * (kTT * 16);         // [64][NP]
+        const int my_rows = max(0, min(rows_per, kTT - rank * rows_per));
+        if (et == 0) {
+          mbar_expect_tx(&sh.rs_full[p], (uint32_t)(C * my_rows * NP * 4));
+          mbar_expect_tx(&sh.ag_full[p], (uint32_t)(kTT * NP * 4));
         }
-        float* xch = sXch + p * (kTT * 16);
         if (lane < 16) {
-          float* dst = xch + (16 * q + lane) * NP;
+          const int R = 16 * q + lane, dest = R / rows_per, lrow = R - dest * rows_per;
+          const uint32_t dst = mapa_shared(smem_u32(rs + (rank * rows_per + lrow) * NP), (uint32_t)dest);
+          const uint32_t bar = mapa_shared(smem_u32(&sh.rs_full[p]), (uint32_t)dest);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
             if (k4 * 4 < NP)
-              *reinterpret_cast<float4*>(dst + k4 * 4) =
-                  make_float4(tsum[k4 * 4], tsum[k4 * 4 + 1], tsum[k4 * 4 + 2], tsum[k4 * 4 + 3]);
+              st_async_f4(dst + k4 * 16, make_float4(tsum[k4 * 4], tsum[k4 * 4 + 1], tsum[k4 * 4 + 2], tsum[k4 * 4 + 3]),
+                          bar);
         }
-        named_bar_sync(1 + grp, 128);
-        if (et < C) mbar_arrive_cluster(mapa_shared(smem_u32(&sh.xch_full[p]), (uint32_t)et));   // one peer per thread
-        ok = mbar_wait_cluster(&sh.xch_full[p], u2 & 1);
+        ok = mbar_wait_cluster(&sh.rs_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        // T = sum over the cluster's partials in rank order; thread = (token row, half of the NP values)
-        const int row = 16 * q + (lane & 15), kh = (lane >> 4) * hn;
-        float acc[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-        const uint32_t mine = smem_u32(xch + row * NP + kh);
         {
-          // all loads first (they are independent), then the sum in rank order
-          float4 va[8], vb[8];
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            va[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-            vb[c] = va[c];
-            if (c < C) {
-              const uint32_t ra = mapa_shared(mine, (uint32_t)c);
-              va[c] = ld_cluster_f4(ra);
-              if (hn == 8) vb[c] = ld_cluster_f4(ra + 16);
+          const int q4 = NP >> 2;                 // float4 pieces per row
+          for (int u = et; u < my_rows * q4; u += 128) {
+            const int lrow = u / q4, k4 = u - lrow * q4;
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c = 0; c < C; ++c) {
+              const float4 v = *reinterpret_cast<const float4*>(rs + (c * rows_per + lrow) * NP + 4 * k4);
+              sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
             }
-          }
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            if (c < C) {
-              acc[0] += va[c].x; acc[1] += va[c].y; acc[2] += va[c].z; acc[3] += va[c].w;
-              acc[4] += vb[c].x; acc[5] += vb[c].y; acc[6] += vb[c].z; acc[7] += vb[c].w;
-            }
+            const uint32_t off = smem_u32(ag + (rank * rows_per + lrow) * NP + 4 * k4);
+            const uint32_t bar = smem_u32(&sh.ag_full[p]);
+            for (int c = 0; c < C; ++c) st_async_f4(mapa_shared(off, (uint32_t)c), sum, mapa_shared(bar, (uint32_t)c));
           }
         }
-        named_bar_sync(1 + grp, 128);        // every thread of the group has finished reading the peers
-        if (et < C) mbar_arrive_cluster(mapa_shared(smem_u32(&sh.xch_free[p]), (uint32_t)et));
+        ok = mbar_wait_cluster(&sh.ag_full[p], u2 & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        // thread = (token row, half of the NP values of T)
+        const int row = 16 * q + (lane & 15), kh = (lane >> 4) * hn;
+        float acc[8];
+        {
+          const float4 a = *reinterpret_cast<const float4*>(ag + row * NP + kh);
+          acc[0] = a.x; acc[1] = a.y; acc[2] = a.z; acc[3] = a.w;
+          float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (hn == 8) b = *reinterpret_cast<const float4*>(ag + row * NP + kh + 4);
+          acc[4] = b.x; acc[5] = b.y; acc[6] = b.z; acc[7] = b.w;
+        }
         // T operand of phase C: rows = hi parts 0..NP-1 then lo parts, 64 tokens (128 bytes) per row
         if (u2 > 0) {
           ok = mbar_wait(&sh.tt_empty[p], (u2 - 1) & 1);
@@ -385,9 +392,9 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
 int g_max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // per cluster size, filled on first use
 
 size_t fz_smem_bytes(int ring) {
-  return (size_t)ring * kSlotBytes + 8 * 32 * 128 + 2 * 32 * 128 + 2 * kTT * 16 * 4 + 1024;
+  return (size_t)ring * kSlotBytes + 8 * 32 * 128 + 2 * 32 * 128 + 2 * kRsFloats * 4 + 2 * kTT * 16 * 4 + 1024;
 }
-constexpr int kFzRing = 11;
+constexpr int kFzRing = 10;
 
 }  // namespace
 

@@ -215,6 +215,13 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t remote_addr) {
                : "r"(remote_addr));
   return v;
 }
+// one-way store of four floats into the shared memory of a CTA of the cluster; the bytes are
+// counted on that CTA's mbarrier (complete_tx), which is how the receiver learns they have landed
+__device__ __forceinline__ void st_async_f4(uint32_t remote_addr, float4 v, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(remote_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar)
+               : "memory");
+}
 // every thread of every CTA of the cluster
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
