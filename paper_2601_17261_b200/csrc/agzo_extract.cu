@@ -182,7 +182,13 @@ __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __rest
     double acc = 0.0;
     const float* yi = sY + i * kGramCols;
     const float* yj = sY + j * kGramCols;
-    for (int c = 0; c < kGramCols; ++c) acc = fma((double)yi[c], (double)yj[c], acc);
+    // rows are 128 floats apart, so all rows share a bank at equal c: every lane starts at its own
+    // column (a fixed rotation, so the sum is still the same on every run)
+    const int rot = threadIdx.x & 31;
+    for (int c = 0; c < kGramCols; ++c) {
+      const int cc = (c + rot) & (kGramCols - 1);
+      acc = fma((double)yi[cc], (double)yj[cc], acc);
+    }
     out[i * r + j] = acc;
   }
 }
@@ -191,8 +197,9 @@ __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __rest
 // S = sum of partial Gram matrices; Cholesky S = R^T R (upper R, positive diagonal); a pivot
 // with R_kk <= kRankTol * R_11 marks a deficient column, which becomes zero.  M (upper
 // triangular) is built so that Q = Y M: column k of M solves R-columns by forward substitution.
-__global__ void __launch_bounds__(64) chol_kernel(const DevLayer* __restrict__ layers, int l0,
-                                                  DevStatus* status) {
+constexpr int kCholThreads = 256;
+__global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __restrict__ layers, int l0,
+                                                            DevStatus* status) {
   const DevLayer& L = layers[l0 + blockIdx.x];
   const int r = L.r;
   __shared__ double S[AGZO_MAX_RANK][AGZO_MAX_RANK + 1];
@@ -200,11 +207,12 @@ __global__ void __launch_bounds__(64) chol_kernel(const DevLayer* __restrict__ l
   __shared__ double piv;
   double* Mm = L.M;                     // [r][r], written and re-read by this block only
   const int tid = threadIdx.x;
-  for (int p = tid; p < r * r; p += 64) {
+  const int ti = tid >> 4, tj = tid & 15;          // 16 x 16 arrangement for the trailing update
+  for (int p = tid; p < r * r; p += kCholThreads) {
     const int i = p / r, j = p - i * r;
     double acc = 0.0;
     if (j >= i)
-      for (int c = 0; c < L.gchunks; ++c) acc += L.Gpart[(long long)c * r * r + p];
+      for (int c = 0; c < L.gchunks; ++c) acc += L.Gpart[(long long)c * r * r + p];   // fixed order
     S[i][j] = acc;
     Mm[p] = 0.0;
   }
@@ -224,12 +232,12 @@ __global__ void __launch_bounds__(64) chol_kernel(const DevLayer* __restrict__ l
     }
     __syncthreads();
     const double pk = piv;
-    for (int j = k + 1 + tid; j < r; j += 64) S[k][j] = pk > 0.0 ? S[k][j] / pk : 0.0;
+    for (int j = k + 1 + tid; j < r; j += kCholThreads) S[k][j] = pk > 0.0 ? S[k][j] / pk : 0.0;
     __syncthreads();
-    const int nn = r - k - 1;
-    for (int p = tid; p < nn * nn; p += 64) {
-      const int i = k + 1 + p / nn, j = k + 1 + p % nn;
-      if (j >= i) S[i][j] -= S[k][i] * S[k][j];
+    for (int i = k + 1 + ti; i < r; i += 16) {
+      const double ski = S[k][i];
+      for (int j = k + 1 + tj; j < r; j += 16)
+        if (j >= i) S[i][j] -= ski * S[k][j];
     }
     __syncthreads();
   }
@@ -237,7 +245,7 @@ __global__ void __launch_bounds__(64) chol_kernel(const DevLayer* __restrict__ l
   // a deficient column stays zero
   for (int k = 0; k < r; ++k) {
     if (!bad[k]) {
-      for (int row = tid; row <= k; row += 64) {
+      for (int row = tid; row <= k; row += kCholThreads) {
         double acc = row == k ? 1.0 : 0.0;
         for (int i = row; i < k; ++i) acc -= Mm[row * r + i] * S[i][k];
         Mm[row * r + k] = acc / S[k][k];
@@ -287,7 +295,7 @@ cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStrea
       w.d_layers, w.l0);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  chol_kernel<<<nl, 64, 0, s>>>(w.d_layers, w.l0, d_status);
+  chol_kernel<<<nl, kCholThreads, 0, s>>>(w.d_layers, w.l0, d_status);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   apply_kernel<<<dim3((w.max_din + 127) / 128, nl), 128, (size_t)w.max_r * w.max_r * sizeof(double), s>>>(
