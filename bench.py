@@ -213,6 +213,7 @@ def main():
     ap.add_argument("--rmw-slots", type=int, default=0)
     ap.add_argument("--rmw-inflight", type=int, default=0)
     ap.add_argument("--rmw-panels", type=int, default=0)
+    ap.add_argument("--rmw-stage-r", type=int, default=0)
     ap.add_argument("--blocks", type=int, default=0,
                     help="keep only the first N transformer blocks of the layer set (profiling-sized runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -254,6 +255,7 @@ def main():
     B.agzo_set_option(ctx, "rmw_tc_slots", args.rmw_slots)
     B.agzo_set_option(ctx, "rmw_tc_inflight", args.rmw_inflight)
     B.agzo_set_option(ctx, "rmw_tc_panels", args.rmw_panels)
+    B.agzo_set_option(ctx, "rmw_stage_r", args.rmw_stage_r)
     if args.wave_mb >= 0:
         B.agzo_set_option(ctx, "wave_bytes", args.wave_mb << 20)
     work = algorithmic_work(cfg, r, args.alias_inputs)
@@ -287,8 +289,9 @@ def main():
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
-    if B.agzo_poll(ctx) not in (B.AGZO_OK,):
-        raise SystemExit("device status not ok after warm-up")
+    st_warm = B.agzo_poll(ctx)
+    if st_warm != B.AGZO_OK:
+        raise SystemExit("device status after warm-up: " + B.status_string(st_warm))
     tc_used = args.extract_path != 1
     dom_class = B.KC_TC_XT_T if tc_used else B.KC_XT_T
     B.agzo_read_counters(ctx)

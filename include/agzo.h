@@ -126,7 +126,10 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * everything else the CUDA-core kernels), 1 = CUDA-core kernels only, 2 = tensor-core kernel
  * for every layer that allows it; tuning knobs of that kernel, 0 = chosen by rank:
  * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),
- * "rmw_tc_panels" (column panels per work item, 1 or 2);
+ * "rmw_tc_panels" (column panels per work item, 1 or 2); "rmw_stage_r" 0 = when some layer's rank
+ * exceeds 16 the split R operand of every 128-row tile is written once per pass to the scratch
+ * area (d_out x 8 r' bytes per layer, r' = r rounded up to 8) and copied in by the pass instead of
+ * being regenerated for every column panel, 1 = never, 2 = always;
  * "share_inputs" 1 (default) = consecutive layers whose X is the same buffer (same pointer, pitch,
  * m, d_in: q/k/v or gate/up of a transformer block) are served by one sweep over X per product,
  * with identical results; 0 = every layer sweeps its X itself;

@@ -1,5 +1,6 @@
 // C ABI of the AGZO library: context, host-side validation, workspace planning and the
 // sequencing of Algorithm 1 / Algorithm 2 over the grouped kernels.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -35,6 +36,9 @@ struct Plan {
   std::vector<int> item_start;
   int total_items = 0;
   int max_rp = 0;
+  bool staged_r = false;           // the tensor-core pass copies R tiles that a fill kernel wrote to scratch
+  int max_row_tiles = 0;
+  size_t image_bytes = 0;
 };
 
 struct PlanOpts {
@@ -43,6 +47,7 @@ struct PlanOpts {
   int rmw_path;          // 0 auto, 1 CUDA-core only, 2 tensor cores wherever a layer allows it
   int rmw_tc_min_rank;   // auto: layers with r >= this use the tensor-core pass
   int rmw_tc_panels;     // column panels per work item of the tensor-core pass (1 or 2)
+  int rmw_stage_r;       // 0: stage R in scratch when some rank exceeds 16; 1: never; 2: always
   bool tc_available;
   bool extract_fused;    // power steps of eligible layers run in the fused single-pass kernel
   bool share_inputs;     // consecutive layers with the same X are served by one sweep
@@ -65,6 +70,7 @@ struct agzo_ctx {
   int rmw_tc_slots;        // ring slots of the tensor-core pass, 0 = as many as fit
   int rmw_tc_inflight;     // loads in flight per CTA, 0 = by rank
   int rmw_tc_panels;       // column panels per work item (1 or 2), 0 = by rank
+  int rmw_stage_r;         // 0 auto, 1 never, 2 always
   int64_t wave_bytes;
   int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
   int extract_fused;       // 1: fused power-step kernel where a layer's shape allows it
@@ -230,6 +236,29 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   int real_waves = 0;
   size_t max_wave_scratch = 0;
 
+  // Which layers take the tensor-core pass, and whether their R operands are staged in scratch
+  // (ranks above 16): the operand image of every 128-row tile of every such layer, laid out from
+  // the start of the scratch area (which extraction uses at other times).
+  auto takes_tc_rmw = [&](const agzo_layer& a) {
+    return tc_available && opts.rmw_path != 1 && rmw_tc_eligible(a) &&
+           (opts.rmw_path == 2 || a.r >= opts.rmw_tc_min_rank);
+  };
+  {
+    size_t img = 0;
+    int max_tiles = 0, max_rp_all = 0;
+    for (int i = 0; i < n; ++i) {
+      if (!takes_tc_rmw(L[i])) continue;
+      img += rmw_tc_image_bytes(L[i]);
+      max_tiles = std::max(max_tiles, (L[i].d_out + 127) / 128);
+      max_rp_all = std::max(max_rp_all, (L[i].r + 7) & ~7);
+    }
+    const size_t room = ws ? (ws_bytes > base ? ws_bytes - base : 0) : (size_t)-1;
+    const bool want = opts.rmw_stage_r == 2 || (opts.rmw_stage_r == 0 && max_rp_all > 16);
+    plan->staged_r = want && img > 0 && img <= room;
+    plan->max_row_tiles = max_tiles;
+    plan->image_bytes = want ? img : 0;
+  }
+  size_t img_off = 0;
   int tiles = 0;
   long long items = 0;
   for (int i = 0; i < n; ++i) {
@@ -247,11 +276,15 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
     if (a.W16) vec = vec && aligned16(a.W16) && (a.ldw16 * 2) % 16 == 0;
     D.vec_ok = vec ? 1 : 0;
     // bf16 weights of sufficient rank go through the tensor-core pass and get no CUDA-core tiles
-    const bool tc_rmw = tc_available && opts.rmw_path != 1 && rmw_tc_eligible(a) &&
-                        (opts.rmw_path == 2 || a.r >= opts.rmw_tc_min_rank);
+    const bool tc_rmw = takes_tc_rmw(a);
     plan->item_start[i] = (int)items;
     if (tc_rmw) {
-      rmw_tc_shape(a, opts.rmw_tc_panels, &D);
+      rmw_tc_shape(a, opts.rmw_tc_panels, plan->staged_r, &D);
+      if (plan->staged_r && ws) {
+        D.rimg = reinterpret_cast<unsigned char*>(ws + base + img_off);
+        D.rimg_tile_bytes = (int)(rmw_tc_image_bytes(a) / (size_t)((a.d_out + 127) / 128));
+      }
+      img_off += rmw_tc_image_bytes(a);
       D.rtc_item0 = (int)items;
       items += (long long)D.rtc_panels * D.rtc_chunks;
       if (items > 0x7fffffff) return AGZO_ERR_INVALID_ARG;
@@ -354,7 +387,10 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
     plan->wave_region.push_back(region);
     i = j;
   }
-  if (scratch_needed) *scratch_needed = max_wave_scratch * regions + (regions > 1 ? kAlign : 0);
+  if (scratch_needed) {
+    *scratch_needed = max_wave_scratch * regions + (regions > 1 ? kAlign : 0);
+    if (plan->image_bytes > *scratch_needed) *scratch_needed = plan->image_bytes;
+  }
   return AGZO_OK;
 }
 
@@ -376,7 +412,7 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (same_layers(c, L, n)) return AGZO_OK;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
-  PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels,
+  PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels, c->rmw_stage_r,
                 c->tc.available, c->extract_fused != 0, c->share_inputs != 0, c->extract_streams};
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
@@ -438,8 +474,9 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   st = prepare(c, L, n, s);
   if (st != AGZO_OK) return st;
   if (c->plan.total_items > 0) {
-    Timed t(c, AGZO_KC_RMW_TC, s);
-    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->rmw_tc_slots, c->rmw_tc_inflight, seed,
+    Timed t(c, AGZO_KC_RMW_TC, s, c->plan.staged_r ? 2 : 1);
+    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->plan.max_row_tiles, c->plan.staged_r,
+                        c->rmw_tc_slots, c->rmw_tc_inflight, seed,
                         coef, d_coef, dev_status(c), c->sm_count, s));
   }
   if (c->plan.total_tiles > 0) {
@@ -481,9 +518,9 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 1, 0, 1, true, false, false, 2}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 8, 0, 0, true, false, false, 2}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, false, false, false, 2}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, false, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -512,6 +549,7 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->rmw_tc_slots = 0;
   c->rmw_tc_inflight = 0;
   c->rmw_tc_panels = 0;
+  c->rmw_stage_r = 0;
   c->wave_bytes = kDefaultWaveBytes;
   c->extract_streams = 2;
   c->extract_fused = 0;
@@ -584,6 +622,9 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
     if (value < 0 || value > 64) return AGZO_ERR_INVALID_ARG;
     ctx->rmw_tc_inflight = (int)value;
     return AGZO_OK;
+  } else if (std::strcmp(name, "rmw_stage_r") == 0) {
+    if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
+    ctx->rmw_stage_r = (int)value;
   } else if (std::strcmp(name, "rmw_tc_panels") == 0) {
     if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
     ctx->rmw_tc_panels = (int)value;

@@ -128,9 +128,43 @@ __device__ __forceinline__ void put_group(uint8_t* base, int atom_bytes, int row
   }
 }
 
+// Rank indices 8g .. 8g+7 of row `row` of R (d_out x r, i.i.d. N(0,1) from the Philox stream
+// (seed, layer_id, tag 0), element e = row * r + k), as bf16 hi parts and bf16 lo parts; zero
+// beyond the matrix.
+__device__ __forceinline__ void gen_r_group(const DevLayer& L, long long row, int g, uint64_t seed, uint4* hi_out,
+                                            uint4* lo_out) {
+  const int r = L.r;
+  const int nv = row < L.d_out ? min(8, r - 8 * g) : 0;   // live rank indices of this group
+  float v[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) v[u] = 0.f;
+  if (nv > 0) {
+    // elements e_first .. e_first + nv - 1 of the stream: at most three Philox blocks
+    const long long e_first = row * r + 8 * g;
+    const long long b0 = e_first >> 2;
+    const int off = (int)(e_first & 3);
+    const int nblk = (off + nv + 3) >> 2;
+    float x[12];
+    const float4 ga = gaussian_block((uint64_t)b0, L.layer_id, kTagG, seed);
+    x[0] = ga.x; x[1] = ga.y; x[2] = ga.z; x[3] = ga.w;
+    float4 gb = make_float4(0.f, 0.f, 0.f, 0.f), gc = gb;
+    if (nblk > 1) gb = gaussian_block((uint64_t)(b0 + 1), L.layer_id, kTagG, seed);
+    if (nblk > 2) gc = gaussian_block((uint64_t)(b0 + 2), L.layer_id, kTagG, seed);
+    x[4] = gb.x; x[5] = gb.y; x[6] = gb.z; x[7] = gb.w;
+    x[8] = gc.x; x[9] = gc.y; x[10] = gc.z; x[11] = gc.w;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const float y = off == 0 ? x[u] : off == 1 ? x[u + 1] : off == 2 ? x[u + 2] : x[u + 3];
+      v[u] = u < nv ? y : 0.f;
+    }
+  }
+  split8(v, hi_out, lo_out);
+}
+
 __global__ void __launch_bounds__(kMaxThreads, 1)
 rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_start, int n_layers,
-              int total_items, int a_bufs, int a_buf_bytes, int slots, int inflight, uint64_t seed, float coef_imm,
+              int total_items, int a_bufs, int a_buf_bytes, int slots, int inflight, int staged, uint64_t seed,
+              float coef_imm,
               const float* __restrict__ d_coef, DevStatus* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -149,7 +183,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
       mbar_init(&sh.empty_w[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&sh.a_full[b], gen_warps);
+      mbar_init(&sh.a_full[b], staged ? 1 : gen_warps);   // staged R: one arrive that sets the byte count
       mbar_init(&sh.a_empty[b], 1);
       mbar_init(&sh.tmem_full[b], 1);
       mbar_init(&sh.tmem_empty[b], kNumEpiWarps);
@@ -261,6 +295,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
     // consecutive rows, so every thread has one or two short independent chains to run.
     const int gt = threadIdx.x - kWarpGen0 * 32;
     int t = 0, ic = 0;
+    int last_ab = -1, last_par = 0;      // the bulk copy this thread issued last (staged R)
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++ic) {
       const Item it = decode_item(layers, item_start, n_layers, item);
@@ -300,35 +335,18 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
           if (!ok) break;
         }
         uint8_t* a_base = sA + (size_t)ab * a_buf_bytes;
+        if (staged) {          // the tile's operand image was written by the fill kernel: one bulk copy
+          if (gt == 0) {
+            mbar_expect_tx(&sh.a_full[ab], (uint32_t)L.rimg_tile_bytes);
+            bulk_load(a_base, L.rimg + (size_t)rb * L.rimg_tile_bytes, (uint32_t)L.rimg_tile_bytes, &sh.a_full[ab]);
+            last_ab = ab; last_par = au & 1;
+          }
+          continue;
+        }
         for (int unit = gt; unit < kRows * g8; unit += gen_threads) {
           const int g = unit >> 7, i = unit & (kRows - 1);
-          const long long row = (long long)rb * kRows + i;
-          const int nv = row < L.d_out ? min(8, r - 8 * g) : 0;   // live rank indices of this group
-          float v[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) v[u] = 0.f;
-          if (nv > 0) {
-            // elements e_first .. e_first + nv - 1 of the stream: at most three Philox blocks
-            const long long e_first = row * r + 8 * g;
-            const long long b0 = e_first >> 2;
-            const int off = (int)(e_first & 3);
-            const int nblk = (off + nv + 3) >> 2;
-            float x[12];
-            const float4 ga = gaussian_block((uint64_t)b0, L.layer_id, kTagG, seed);
-            x[0] = ga.x; x[1] = ga.y; x[2] = ga.z; x[3] = ga.w;
-            float4 gb = make_float4(0.f, 0.f, 0.f, 0.f), gc = gb;
-            if (nblk > 1) gb = gaussian_block((uint64_t)(b0 + 1), L.layer_id, kTagG, seed);
-            if (nblk > 2) gc = gaussian_block((uint64_t)(b0 + 2), L.layer_id, kTagG, seed);
-            x[4] = gb.x; x[5] = gb.y; x[6] = gb.z; x[7] = gb.w;
-            x[8] = gc.x; x[9] = gc.y; x[10] = gc.z; x[11] = gc.w;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const float y = off == 0 ? x[u] : off == 1 ? x[u + 1] : off == 2 ? x[u + 2] : x[u + 3];
-              v[u] = u < nv ? y : 0.f;
-            }
-          }
           uint4 hi, lo;
-          split8(v, &hi, &lo);
+          gen_r_group(L, (long long)rb * kRows + i, g, seed, &hi, &lo);
           put_group(a_base, kAtomBytesA, i, g, g8, hi, lo, 0, 1, 2, 3);
         }
         fence_proxy_async();
@@ -337,6 +355,8 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
       }
     }
     if (!ok) sh.failed = 1;
+    // leaving early with a bulk copy in flight: it must land before the CTA goes away
+    if (staged && gt == 0 && last_ab >= 0 && (!ok || sh.failed)) mbar_wait(&sh.a_full[last_ab], (uint32_t)last_par);
   } else {
     // ------------------------------------------------ epilogue: thread = row of the tile, 32 columns of each box
     const int e = warp - kWarpEpi0;
@@ -401,6 +421,24 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
   if (warp == kWarpMma) { tc_fence_after(); tmem_dealloc(tmem, kTmemCols); }
 }
 
+// Staged R: CTA = (row tile, layer); writes the tile's split A operand [Rh | Rh | Rl | Rl] to
+// scratch exactly as rmw_tc_kernel lays it out in shared memory (K atoms of [128 rows][128 bytes],
+// 128-byte swizzle), so the pass can bulk-copy it.
+__global__ void __launch_bounds__(256) rmw_tc_fill_r_kernel(const DevLayer* __restrict__ layers, uint64_t seed) {
+  const DevLayer& L = layers[blockIdx.y];
+  if (!L.rimg) return;
+  const int rb = blockIdx.x;
+  if (rb * kRows >= L.d_out) return;
+  const int g8 = L.rtc_rp >> 3;
+  uint8_t* img = L.rimg + (size_t)rb * L.rimg_tile_bytes;
+  for (int unit = threadIdx.x; unit < kRows * g8; unit += 256) {
+    const int g = unit >> 7, i = unit & (kRows - 1);
+    uint4 hi, lo;
+    gen_r_group(L, (long long)rb * kRows + i, g, seed, &hi, &lo);
+    put_group(img, kAtomBytesA, i, g, g8, hi, lo, 0, 1, 2, 3);
+  }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------- host side
@@ -409,19 +447,25 @@ bool rmw_tc_eligible(const agzo_layer& a) {
          (a.ldw * 2) % 16 == 0 && a.d_out >= 1 && a.d_in >= 1 && a.r >= 1 && a.r <= AGZO_MAX_RANK;
 }
 
-void rmw_tc_shape(const agzo_layer& a, int panels, DevLayer* D) {
+void rmw_tc_shape(const agzo_layer& a, int panels, bool staged, DevLayer* D) {
   const int rp = (a.r + 7) & ~7;
   const int katoms = (4 * rp + 63) / 64;                 // 1, 2, 3 or 4 K atoms of 64
-  const int cw = katoms == 1 ? 256 : katoms == 2 ? 128 : 64;
+  // Panel width: K atoms x columns x 128 bytes of B operand must fit its area (32 KiB per panel,
+  // 64 KiB when one panel takes both).  With R staged in scratch there is nothing to amortise over
+  // a second panel, so one wide panel is used (fewer, larger MMAs).
+  const int cw = katoms == 1 ? 256 : staged ? (katoms == 2 ? 256 : 128) : (katoms == 2 ? 128 : 64);
   // panels == 0: one panel per item while R is cheap to regenerate (rp <= 16: the pass is
   // HBM-bound either way and the smaller items balance better), two from there on, where
   // regenerating R is what limits the pass
-  const int np = panels == 1 ? 1 : panels == 2 ? kMaxPanels : (katoms == 1 ? 1 : kMaxPanels);
+  int np = panels == 1 ? 1 : panels == 2 ? kMaxPanels : (katoms == 1 ? 1 : kMaxPanels);
+  if (staged && katoms >= 2) np = 1;
   D->rtc_rp = rp;
   D->rtc_cw = cw;
   D->rtc_np = np;
   D->rtc_panels = (a.d_in + np * cw - 1) / (np * cw);   // panel groups
-  D->rtc_chunk_blocks = 8;
+  // row tiles per item: the B operand is rebuilt once per item, which stalls the MMA pipeline for a
+  // few microseconds when the rank is large, so those items are taller
+  D->rtc_chunk_blocks = katoms >= 2 ? 32 : 8;
   const int nrb = (a.d_out + kRows - 1) / kRows;
   D->rtc_chunks = (nrb + D->rtc_chunk_blocks - 1) / D->rtc_chunk_blocks;
 }
@@ -436,13 +480,26 @@ cudaError_t rmw_tc_init() {
   return cudaFuncSetAttribute(rmw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
 }
 
+size_t rmw_tc_image_bytes(const agzo_layer& a) {
+  const int rp = (a.r + 7) & ~7;
+  const size_t katoms = (size_t)(4 * rp + 63) / 64;
+  return (size_t)((a.d_out + kRows - 1) / kRows) * katoms * kAtomBytesA;
+}
+
 cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
-                          int max_rp, int slots_wanted, int inflight, uint64_t seed, float coef, const float* d_coef,
-                          DevStatus* d_status, int sm_count, cudaStream_t s) {
+                          int max_rp, int max_row_tiles, bool staged, int slots_wanted, int inflight, uint64_t seed,
+                          float coef, const float* d_coef, DevStatus* d_status, int sm_count, cudaStream_t s) {
   if (total_items <= 0) return cudaSuccess;
+  if (staged) {
+    rmw_tc_fill_r_kernel<<<dim3((unsigned)max_row_tiles, (unsigned)n_layers), 256, 0, s>>>(d_layers, seed);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
   const int katoms = (4 * max_rp + 63) / 64;
   const int a_buf_bytes = katoms * kAtomBytesA;
-  const int a_bufs = katoms >= 3 ? 1 : 2;
+  // one A buffer where two would leave too few ring slots; with staged R the buffer is refilled by a
+  // bulk copy that is short next to the tile's HBM time
+  const int a_bufs = (katoms >= 3 || (staged && katoms >= 2)) ? 1 : 2;
   const int fixed = a_bufs * a_buf_bytes + kMaxPanels * kBBytes;
   int slots = (224 * 1024 - fixed) / kBoxBytes;
   if (slots > kMaxSlots) slots = kMaxSlots;
@@ -456,7 +513,7 @@ cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int
   if (inflight < 1) inflight = max_rp <= 8 ? 4 : 5;
   if (inflight > slots) inflight = slots;
   rmw_tc_kernel<<<grid, threads, smem, s>>>(d_layers, d_item_start, n_layers, total_items, a_bufs, a_buf_bytes,
-                                             slots, inflight, seed, coef, d_coef, d_status);
+                                             slots, inflight, staged ? 1 : 0, seed, coef, d_coef, d_status);
   return cudaGetLastError();
 }
 

@@ -120,6 +120,28 @@ def test_perturb_restore_update_match_oracle(d_out, d_in, r, storage, extra, lab
         assert bool((Vbuf[0] == 7).all() and (Vbuf[:, d_in:] == 7).all())
 
 
+@pytest.mark.parametrize("stage", [1, 2])
+def test_tensor_core_pass_with_and_without_staged_R(stage):
+    # stage 2: R tiles written to scratch by a fill kernel even at r = 8; stage 1: regenerated in the pass at r = 40
+    d_out, d_in, r = (300, 640, 8) if stage == 2 else (300, 384, 40)
+    seed, layer_id = 4, 2
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=8, bf16=True)
+    Vh = O.extract_subspace(WL.plain_activations(2 * r + 16, d_in, seed=r), r, 1, 3, layer_id)
+    Wd, _ = to_dev(W0, True)
+    Vd, _ = to_dev(Vh, False)
+    layers = [B.make_layer(W=Wd, V=Vd, r=r, layer_id=layer_id)]
+    with Ctx(layers, extra=1 << 20) as ctx:
+        B.agzo_set_option(ctx, "rmw_path", 2)
+        B.agzo_set_option(ctx, "rmw_stage_r", stage)
+        for c in (1e-3, -2e-3):
+            before = to_host(Wd)
+            B.agzo_perturb(ctx, layers, seed, c)
+            want = O.apply_direction(before, Vh, seed, layer_id, np.float32(c), "bf16")
+            assert_weights_match(to_host(Wd), want, "bf16",
+                                 floor=cancellation_floor(before, c, seed, layer_id, Vh, rel=2.0 ** -16))
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+
+
 def test_restore_update_fused_modes():
     d_out, d_in, r, seed = 200, 512, 8, 21
     W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=1, bf16=True)
