@@ -383,6 +383,12 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       j += glen;
     }
     if (used > max_wave_scratch) max_wave_scratch = used;
+    {   // order in which T = X Q takes the wave's layers: largest d_in first (stable)
+      std::vector<int> ord(j - i);
+      for (int k = 0; k < j - i; ++k) ord[k] = k;
+      std::stable_sort(ord.begin(), ord.end(), [&](int a, int b) { return L[i + a].d_in > L[i + b].d_in; });
+      for (int k = 0; k < j - i; ++k) plan->dev[i + k].xq_order = ord[k];
+    }
     plan->wave_end.push_back(j);
     plan->wave_region.push_back(region);
     i = j;

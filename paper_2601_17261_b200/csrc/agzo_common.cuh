@@ -38,6 +38,7 @@ struct alignas(16) DevLayer {
   const void* tmaps;     // four 128-byte TMA descriptors of this layer: X, Qb, Tb, unused
   long long m_pad;       // row pitch of Tb in elements (m rounded up to 8)
   int NB, NP;
+  int xq_order;          // T = X Q: the CTA row of this wave position works on layer (wave start + xq_order), longest rows first
   int fz_C;              // cluster size of the fused power-step kernel for this layer, 0 = unfused kernels
   // Consecutive layers that read the same X (q/k/v, gate/up of a transformer block) form a group:
   // their operand panels are adjacent rows of one matrix, the leader's CTAs run both products

@@ -56,7 +56,10 @@ __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16* hi, __nv_bflo
 // One CTA per 128-token tile of one layer.  grid = (max token tiles, layers in the wave).
 __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __restrict__ layers, int l0,
                                                             DevStatus* status, int stages, int skip_fused) {
-  const DevLayer& L = layers[l0 + blockIdx.y];
+  // CTA rows are handed out in the order the scheduler starts them: the layers with the longest
+  // token rows (largest d_in, longest CTAs) go first so that the wave does not end on them
+  const int li = l0 + layers[l0 + blockIdx.y].xq_order;
+  const DevLayer& L = layers[li];
   const int t0 = blockIdx.x * 128;
   if (t0 >= L.m || (skip_fused && L.fz_C) || L.grp_role == 2) return;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -130,7 +133,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
     const int t = t0 + q * 32 + lane;
     if (ok) {
       for (int mi = 0; mi < nmem; ++mi) {               // the layers this CTA serves
-        const DevLayer& M = layers[l0 + blockIdx.y + mi];
+        const DevLayer& M = layers[li + mi];
         const int NP = M.NP, off = L.grp_role == 1 ? M.grp_off : 0;
         __nv_bfloat16* Tt = M.Tb;
         const long long mp = M.m_pad;
