@@ -65,3 +65,59 @@ def test_in_place_passes_on_a_full_size_layer(d_out, d_in, r):
         assert_weights_match(to_host(Wd), want, "bf16", frac=frac,
                              floor=cancellation_floor(cur, c, seed, layer_id, Vh, rel))
         assert B.agzo_poll(ctx) == B.AGZO_OK
+
+
+def test_every_layer_of_the_0p6b_shaped_set_in_one_grouped_launch():
+    """All 196 layers of the Qwen3-0.6B-shaped set (0.44 G bf16 weights) perturbed by one call, every
+    weight compared with the oracle; the layer shapes repeat per block, so the directions are
+    computed per distinct (layer_id, shape) as the library sees them."""
+    cfg = WL.QWEN3_0P6B
+    r, seed, eps = 8, 11, 1e-3
+    specs = cfg.layers()
+    host_W, dev_W, dev_V, host_V, layers = [], [], [], [], []
+    Vcache = {}
+    for i, (name, d_in, d_out) in enumerate(specs):
+        W0 = WL.gaussian_weights(d_out, d_in, cfg.w_std, seed=1000 + i, bf16=True)
+        if d_in not in Vcache:      # any orthonormal basis will do for the pass; one per input width
+            Vcache[d_in] = O.extract_subspace(WL.plain_activations(64, d_in, seed=d_in), r, 1, 3, 0)
+        Vh = Vcache[d_in]
+        Wd, _ = to_dev(W0, True)
+        Vd, _ = to_dev(Vh, False)
+        host_W.append(W0); host_V.append(Vh); dev_W.append(Wd); dev_V.append(Vd)
+        layers.append(B.make_layer(W=Wd, V=Vd, r=r, layer_id=i))
+    with Ctx(layers) as ctx:
+        B.agzo_perturb(ctx, layers, seed, eps)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    for i in range(len(specs)):
+        want = O.apply_direction(host_W[i], host_V[i], seed, i, np.float32(eps), "bf16")
+        assert_weights_match(to_host(dev_W[i]), want, "bf16",
+                             floor=cancellation_floor(host_W[i], eps, seed, i, host_V[i], 2.0 ** -16))
+
+
+def test_extraction_of_two_blocks_of_the_0p6b_shaped_set_with_shared_inputs():
+    """Blocks 0 and 27 of the Qwen3-0.6B-shaped set in one call, q/k/v and gate/up reading one
+    activation buffer each as in a transformer block."""
+    cfg = WL.QWEN3_0P6B
+    r, K, seed = 8, 3, 4
+    layers, keep, checks = [], [], []
+    for blk in (0, 27):
+        Xq = WL.planted_activations(cfg.m, 1024, cfg.planted_rank, seed=100 + blk, bf16=True)
+        Xo = WL.planted_activations(cfg.m, 2048, cfg.planted_rank, seed=200 + blk, bf16=True)
+        Xg = WL.planted_activations(cfg.m, 1024, cfg.planted_rank, seed=300 + blk, bf16=True)
+        Xd = WL.planted_activations(cfg.m, 3072, cfg.planted_rank, seed=400 + blk, bf16=True)
+        dq, do_, dg, dd = (to_dev(x, True)[0] for x in (Xq, Xo, Xg, Xd))
+        for j, (Xh, Xdev) in enumerate([(Xq, dq), (Xq, dq), (Xq, dq), (Xo, do_), (Xg, dg), (Xg, dg), (Xd, dd)]):
+            lid = 7 * blk + j
+            V = torch.zeros(r, Xh.shape[1], device=DEV)
+            keep.append((Xdev, V))
+            layers.append(B.make_layer(X=Xdev, V=V, r=r, layer_id=lid))
+            checks.append((Xh, V, lid))
+    with Ctx(layers) as ctx:
+        B.agzo_extract_subspace(ctx, layers, seed, K)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    for Xh, V, lid in checks:
+        Vg = to_host(V)
+        Vo = O.extract_subspace(Xh, r, K, seed, lid)
+        assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
+        assert projector_distance(Vg, Vo) <= 1e-3
+        assert np.abs(Vg - Vo).max() <= 1e-3
