@@ -193,10 +193,6 @@ __device__ __forceinline__ uint32_t cluster_count_x() {
 __device__ __forceinline__ uint32_t mapa_shared(uint32_t saddr, uint32_t rank) {
   uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank)); return r;
 }
-// arrive (release at cluster scope) on an mbarrier that lives in another CTA of the cluster
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
-}
 // bounded wait with acquire at cluster scope: for barriers that CTAs of the cluster arrive on
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {
   const unsigned long long t0 = global_ns();
@@ -216,13 +212,6 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     if (global_ns() - t0 > kWaitCapNs) return false;
   }
 }
-__device__ __forceinline__ float4 ld_cluster_f4(uint32_t remote_addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(remote_addr));
-  return v;
-}
 // one-way store of four floats into the shared memory of a CTA of the cluster; the bytes are
 // counted on that CTA's mbarrier (complete_tx), which is how the receiver learns they have landed
 __device__ __forceinline__ void st_async_f4(uint32_t remote_addr, float4 v, uint32_t remote_bar) {
@@ -234,9 +223,6 @@ __device__ __forceinline__ void st_async_f4(uint32_t remote_addr, float4 v, uint
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void named_bar_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 }  // namespace ptx
