@@ -214,6 +214,10 @@ def main():
     ap.add_argument("--rmw-inflight", type=int, default=0)
     ap.add_argument("--rmw-panels", type=int, default=0)
     ap.add_argument("--rmw-stage-r", type=int, default=0)
+    ap.add_argument("--method", default="agzo", choices=["agzo", "lozo", "mezo"],
+                    help="agzo: the benchmarked path.  lozo / mezo: the same library's kernels arranged as those "
+                         "estimators' step (Gaussian right factor instead of extraction; dense Gaussian direction), "
+                         "for a like-for-like step-overhead comparison")
     ap.add_argument("--blocks", type=int, default=0,
                     help="keep only the first N transformer blocks of the layer set (profiling-sized runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -264,7 +268,19 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step(seed: int):
-        B.agzo_extract_subspace(ctx, layers, seed, K_POWER, arr=arr)
+        if args.method == "mezo":      # dense N(0, I) direction on every weight, three passes
+            for i, W in enumerate(Ws):
+                B.agzo_perturb_dense(ctx, W.view(-1), seed, i, EPS)
+            for i, W in enumerate(Ws):
+                B.agzo_perturb_dense(ctx, W.view(-1), seed, i, -2 * EPS)
+            B.agzo_ghat(ctx, losses[0:1], losses[1:2], EPS, 0, ghat)
+            for i, W in enumerate(Ws):
+                B.agzo_perturb_dense(ctx, W.view(-1), seed, i, EPS - LR, d_scale=None)
+            return
+        if args.method == "lozo":      # U V^T with both factors from the seed: no extraction
+            B.agzo_fill_gaussian_basis(ctx, layers, seed, arr=arr)
+        else:
+            B.agzo_extract_subspace(ctx, layers, seed, K_POWER, arr=arr)
         B.agzo_perturb(ctx, layers, seed, EPS, arr=arr)
         B.agzo_perturb(ctx, layers, seed, -2 * EPS, arr=arr)
         B.agzo_ghat(ctx, losses[0:1], losses[1:2], EPS, 0, ghat)
@@ -361,7 +377,7 @@ def main():
             "metric": METRIC, "value": ms_step, "unit": "ms", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic",
-            "data": "synthetic",
+            "data": "synthetic", "method": args.method,
             "config": {"workload": f"{cfg.name}: {len(layers)} layers, {cfg.n_params() / 1e9:.3f} G weights, "
                                    f"m={cfg.m} tokens, r={r}, K={K_POWER}, eps={EPS}, two-point",
                        "l2": "inputs larger than L2 (weights %.1f GB + activations %.1f GB per step)"

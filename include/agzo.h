@@ -31,7 +31,8 @@
  *   - Random streams: Philox4x32-10 with key = the 64-bit step seed and counter
  *     (b_lo, b_hi, layer_id, tag); b = e >> 2 where e is the row-major index of the element
  *     inside the matrix being drawn, which takes output word e & 3 of that block.
- *     tag 0 = R_l (d_out x r), tag 1 = Omega (m x r), tag 2 = dense direction.
+ *     tag 0 = R_l (d_out x r), tag 1 = Omega (m x r), tag 2 = dense direction,
+ *     tag 3 = Gaussian right factor (r x d_in) of the LOZO comparison.
  *     Normals are Box-Muller on the word pairs (x0,x1) and (x2,x3):
  *       u1 = ((x >> 8) + 1) * 2^-24, u2 = (x' >> 8) * 2^-24, s = sqrt(-2 ln u1),
  *       even lane = s*cos(2 pi u2), odd lane = s*sin(2 pi u2), in fp32.
@@ -234,6 +235,14 @@ agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n,
 agzo_status agzo_perturb_dense(agzo_ctx* ctx, void* w, int64_t n_elems, int dtype,
                                uint64_t seed, uint32_t layer_id, float scale,
                                const float* d_scale, void* stream);
+
+/* Data-independent right factor, for comparison runs with LOZO (Section 2, Eq. lozo-layer-perturb:
+ * Delta_l = U_l V_l^T with both factors Gaussian): V_l (stored as r rows of length d_in) is filled
+ * with i.i.d. N(0,1) from (seed, layer_id, tag 3), element e = k * d_in + d.  The in-place passes
+ * then apply U_l V_l^T exactly as they apply R_l A_l^T; LOZO's 1 / r_l belongs in the caller's step
+ * size.  Only V, ldv, r, d_in and layer_id of the descriptors are used.                    */
+agzo_status agzo_fill_gaussian_basis(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                                     void* stream);
 
 /* ---------------------------------------------------------------- allocation-free variant */
 

@@ -42,6 +42,7 @@ _SH32 = np.uint64(32)
 TAG_G = 0        # left factor R_l of Eq. (agzo-perturb)
 TAG_OMEGA = 1    # test matrix Omega of Algorithm 1
 TAG_DENSE = 2    # dense Gaussian direction for non-matrix parameters (Eq. agzo-perturb, case 2)
+TAG_BASIS = 3    # Gaussian right factor V_l of LOZO (Eq. lozo-layer-perturb), for comparison runs
 
 
 def philox4x32_10(c0, c1, c2, c3, k0, k1):
@@ -109,6 +110,11 @@ def gen_G(seed: int, layer_id: int, d_out: int, r: int) -> np.ndarray:
 def gen_omega(seed: int, layer_id: int, m: int, r: int) -> np.ndarray:
     """Gaussian test matrix Omega of Algorithm 1, m x r, float32."""
     return gaussian_stream(seed, layer_id, TAG_OMEGA, m * r).reshape(m, r)
+
+
+def gen_gaussian_basis(seed: int, layer_id: int, r: int, d_in: int) -> np.ndarray:
+    """V_l^T of Eq. (lozo-layer-perturb): r x d_in i.i.d. N(0,1), float32, row-major stream."""
+    return gaussian_stream(seed, layer_id, TAG_BASIS, r * d_in).reshape(r, d_in)
 
 
 def gen_dense(seed: int, layer_id: int, n: int) -> np.ndarray:

@@ -31,7 +31,7 @@ EXPORTS = [
     "agzo_status_string", "agzo_last_cuda_error", "agzo_extract_subspace", "agzo_perturb",
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
-    "agzo_extract_subspace_static",
+    "agzo_extract_subspace_static", "agzo_fill_gaussian_basis",
 ]
 KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC, KC_FUSED_POWER = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
@@ -87,6 +87,7 @@ def lib() -> C.CDLL:
         "agzo_last_cuda_error": (i32, [vp]),
         "agzo_extract_subspace": (i32, [vp, LP, i32, u64, i32, vp]),
         "agzo_perturb": (i32, [vp, LP, i32, u64, f32, vp]),
+        "agzo_fill_gaussian_basis": (i32, [vp, LP, i32, u64, vp]),
         "agzo_restore": (i32, [vp, LP, i32, u64, f32, vp]),
         "agzo_update": (i32, [vp, LP, i32, u64, f32, vp, vp]),
         "agzo_ghat": (i32, [vp, vp, vp, f32, i32, vp, vp]),
@@ -241,6 +242,12 @@ def agzo_extract_subspace_static(X: torch.Tensor, V: torch.Tensor, r: int, K: in
                                               X.shape[1], r, K, seed, layer_id, V.data_ptr(),
                                               V.stride(0), flag, _stream_ptr(stream)),
            "agzo_extract_subspace_static")
+
+
+def agzo_fill_gaussian_basis(ctx: Context, layers, seed: int, stream=None, arr=None) -> None:
+    arr = arr if arr is not None else layer_array(layers)
+    _check(lib().agzo_fill_gaussian_basis(ctx.handle, arr, len(layers), seed, _stream_ptr(stream)),
+           "agzo_fill_gaussian_basis")
 
 
 def agzo_perturb(ctx: Context, layers, seed: int, scale: float, stream=None, arr=None) -> None:

@@ -900,12 +900,30 @@ agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n, const ag
   return agzo_restore_update(ctx, h_layers, n, p->seed, p->eps, p->lr, p->mode, d_g, stream);
 }
 
+agzo_status agzo_fill_gaussian_basis(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
+                                     void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  st = validate(h_layers, n, 0);
+  if (st != AGZO_OK) return st;
+  if (n == 0) return AGZO_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = prepare(ctx, h_layers, n, s);
+  if (st != AGZO_OK) return st;
+  int max_elems = 0;
+  for (int i = 0; i < n; ++i) max_elems = std::max(max_elems, h_layers[i].r * h_layers[i].d_in);
+  ctx->launches += 1;
+  CU(ctx, launch_fill_basis(dev_layers(ctx), n, max_elems, seed, s));
+  return AGZO_OK;
+}
+
 agzo_status agzo_perturb_dense(agzo_ctx* ctx, void* w, int64_t n_elems, int dtype, uint64_t seed,
                                uint32_t layer_id, float scale, const float* d_scale, void* stream) {
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
   if (n_elems < 0 || (n_elems > 0 && !w)) return AGZO_ERR_INVALID_ARG;
   if (dtype != AGZO_BF16 && dtype != AGZO_F32) return AGZO_ERR_UNSUPPORTED;
+  ctx->launches += 1;
   CU(ctx, launch_dense(w, n_elems, dtype, seed, layer_id, scale, d_scale,
                        static_cast<cudaStream_t>(stream)));
   return AGZO_OK;

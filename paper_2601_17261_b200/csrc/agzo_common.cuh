@@ -128,7 +128,7 @@ __device__ __forceinline__ float4 gaussian_block(uint64_t block, uint32_t layer_
   return box_muller4(philox4x32_10(block, layer_id, tag, seed));
 }
 
-constexpr uint32_t kTagG = 0, kTagOmega = 1, kTagDense = 2;
+constexpr uint32_t kTagG = 0, kTagOmega = 1, kTagDense = 2, kTagBasis = 3;
 
 // ---------------------------------------------------------------- launch entry points (host)
 // in-place passes; d_coef != nullptr overrides coef
@@ -138,6 +138,7 @@ cudaError_t launch_rmw(const DevLayer* d_layers, const int* d_tile_start, int n_
                        int sm_count, cudaStream_t s);
 cudaError_t launch_dense(void* w, long long n, int dtype, uint64_t seed, uint32_t layer_id,
                          float scale, const float* d_scale, cudaStream_t s);
+cudaError_t launch_fill_basis(const DevLayer* d_layers, int n_layers, int max_elems, uint64_t seed, cudaStream_t s);
 cudaError_t launch_ghat(const double* fp, const double* fo, float eps, int mode, float* g,
                         cudaStream_t s);
 cudaError_t launch_coef(const float* g, float eps, float lr, int kind, float* d_coef,

@@ -431,6 +431,35 @@ cudaError_t launch_dense(void* w, long long n, int dtype, uint64_t seed, uint32_
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ Gaussian right factor (LOZO comparison)
+__global__ void fill_basis_kernel(const DevLayer* __restrict__ layers, uint64_t seed) {
+  const DevLayer& L = layers[blockIdx.y];
+  const long long n = (long long)L.r * L.d_in;
+  const long long nb = (n + 3) >> 2;
+  for (long long b = blockIdx.x * (long long)blockDim.x + threadIdx.x; b < nb;
+       b += (long long)gridDim.x * blockDim.x) {
+    const float4 g = gaussian_block((uint64_t)b, L.layer_id, kTagBasis, seed);
+    const float gv[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+    for (int lane = 0; lane < 4; ++lane) {
+      const long long e = 4 * b + lane;
+      if (e < n) {
+        const long long k = e / L.d_in;
+        L.V[k * L.ldv + (e - k * L.d_in)] = gv[lane];
+      }
+    }
+  }
+}
+
+cudaError_t launch_fill_basis(const DevLayer* d_layers, int n_layers, int max_elems, uint64_t seed, cudaStream_t s) {
+  if (n_layers <= 0) return cudaSuccess;
+  int gx = (max_elems / 4 + 255) / 256;
+  if (gx < 1) gx = 1;
+  if (gx > 64) gx = 64;
+  fill_basis_kernel<<<dim3((unsigned)gx, (unsigned)n_layers), 256, 0, s>>>(d_layers, seed);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ scalars (Algorithm 2, step 3)
 __global__ void ghat_kernel(const double* fp, const double* fo, float eps, int mode, float* g) {
   const double d = *fp - *fo;

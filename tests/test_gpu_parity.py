@@ -216,6 +216,30 @@ def test_dense_direction():
         assert d.max() <= 1 and (d > 0).mean() < 1e-3
 
 
+def test_gaussian_right_factor_matches_the_oracle_and_feeds_the_passes():
+    specs = [(300, 640, 8), (64, 100, 3)]
+    devs, layers = [], []
+    for i, (do, di, r) in enumerate(specs):
+        W0 = WL.gaussian_weights(do, di, 0.02, seed=30 + i, bf16=True)
+        Wd, _ = to_dev(W0, True)
+        Vbuf = torch.full((r + 2, di + 4), 7.0, device=DEV)
+        devs.append((W0, Wd, Vbuf))
+        layers.append(B.make_layer(W=Wd, V=Vbuf[1:1 + r, :di], r=r, layer_id=50 + i))
+    with Ctx(layers) as ctx:
+        B.agzo_fill_gaussian_basis(ctx, layers, 77)
+        B.agzo_perturb(ctx, layers, 77, 1e-3)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    for i, (do, di, r) in enumerate(specs):
+        W0, Wd, Vbuf = devs[i]
+        Vg = to_host(Vbuf[1:1 + r, :di])
+        Vo = O.gen_gaussian_basis(77, 50 + i, r, di)
+        assert (np.abs(Vg.astype(np.float64) - Vo) / np.maximum(1.0, np.abs(Vo))).max() <= 2e-6
+        assert bool((Vbuf[0] == 7).all() and (Vbuf[-1] == 7).all() and (Vbuf[:, di:] == 7).all())
+        want = O.apply_direction(W0, Vg, 77, 50 + i, np.float32(1e-3), "bf16")     # U V^T with the device's V
+        assert_weights_match(to_host(Wd), want, "bf16",
+                             floor=cancellation_floor(W0, 1e-3, 77, 50 + i, Vg, rel=2.0 ** -16))
+
+
 def test_ghat_scalar():
     V = torch.zeros(1, 8, device=DEV)
     fp = torch.tensor([0.731234], device=DEV, dtype=torch.float64)

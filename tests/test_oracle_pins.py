@@ -393,3 +393,20 @@ def test_gelu_and_mlp_forward_against_torch():
     out16, ins = O.mlp_forward([O.round_bf16(W) for W in Ws], x0, True, collect_inputs=True)
     assert len(ins) == 3 and np.array_equal(ins[0], WL.to_bf16_values(x0))
     assert np.abs(out16 - out).max() < 0.2
+
+
+def test_gaussian_right_factor_of_the_lozo_comparison():
+    """Eq. (lozo-layer-perturb): both factors Gaussian.  The right factor is its own stream (tag 3), laid
+    out as r rows of d_in, independent of the left factor's stream, and U V^T has E||Delta||_F^2 = d_out d_in r."""
+    r, d_in, d_out = 4, 96, 64
+    V = O.gen_gaussian_basis(9, 5, r, d_in)
+    flat = O.gaussian_stream(9, 5, O.TAG_BASIS, r * d_in)
+    assert V.shape == (r, d_in) and np.array_equal(V.reshape(-1), flat)
+    assert not np.array_equal(flat[: d_out * r], O.gen_G(9, 5, d_out, r).reshape(-1)[: r * d_in][: d_out * r])
+    big = O.gen_gaussian_basis(1, 0, 8, 50000)
+    assert abs(big.mean()) < 5e-3 and abs(big.var() - 1.0) < 1e-2
+    tot = 0.0
+    for s in range(200):
+        D = O.lowrank_direction(O.gen_G(s, 0, d_out, r), O.gen_gaussian_basis(s, 0, r, d_in))
+        tot += (D * D).sum()
+    assert abs(tot / 200 / (d_out * d_in * r) - 1.0) < 0.05
