@@ -155,41 +155,99 @@ cudaError_t launch_x_q(const ExtractWave& w, cudaStream_t s) {
 
 // ------------------------------------------------------------------ qr(Y), stage 1
 // Y[k][d] = sum_s Ypart[s][k][d] (fixed order) and the partial Gram matrix of this block's
-// column chunk in double.  block = 128 columns.
+// columns in double.  A block takes kGramGroup chunks of 128 columns one after another and keeps
+// its sums in registers across them: thread = (4 x 4 block of the Gram matrix, part of the
+// columns), so every pair of loaded values feeds 16 multiply-adds.
 constexpr int kGramCols = 128;
+constexpr int kGramGroup = 4;
+__host__ __device__ inline int gram_csplit(int r4) {   // column parts per chunk: as many as 256 threads allow
+  const int nsq = (r4 >> 2) * (r4 >> 2);
+  int cs = 16;
+  while (cs > 1 && cs * nsq > 256) cs >>= 1;
+  return cs;
+}
+__host__ __device__ inline size_t gram_smem_bytes(int r) {
+  const int r4 = (r + 3) & ~3;
+  const size_t y = (size_t)r4 * kGramCols * sizeof(float);
+  const size_t red = (size_t)gram_csplit(r4) * r4 * r4 * sizeof(double);
+  return y > red ? y : red;
+}
+// the launch serves layers of several ranks, and the need is not monotone in r (fewer column
+// parts fit at larger r): take the largest need over all ranks up to the wave's maximum
+inline size_t gram_smem_bytes_upto(int max_r) {
+  size_t b = 0;
+  for (int r = 1; r <= max_r; ++r) b = gram_smem_bytes(r) > b ? gram_smem_bytes(r) : b;
+  return b;
+}
 __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0) {
   const DevLayer& L = layers[l0 + blockIdx.y];
-  const int chunk = blockIdx.x;
-  if (chunk >= L.gchunks) return;
-  extern __shared__ __align__(16) float sY[];   // [r][kGramCols]
-  const int r = L.r;
-  const int d0 = chunk * kGramCols;
-  for (int i = threadIdx.x; i < r * kGramCols; i += 256) {
-    const int k = i / kGramCols, c = i - k * kGramCols;
-    const int d = d0 + c;
-    float y = 0.f;
-    if (d < L.d_in) {
-      for (int s = 0; s < L.slabs; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
-      L.Y[(long long)k * L.d_in + d] = y;
+  const int ngroups = (L.gchunks + kGramGroup - 1) / kGramGroup;
+  const int grp = blockIdx.x;
+  if (grp >= ngroups) return;
+  extern __shared__ __align__(16) unsigned char gram_smem[];
+  float* sY = reinterpret_cast<float*>(gram_smem);        // [r4][kGramCols]; later reused for the column parts' sums
+  const int r = L.r, r4 = (r + 3) & ~3, nb = r4 >> 2;
+  const int csplit = gram_csplit(r4), clen = kGramCols / csplit;
+  const int unit = threadIdx.x;
+  const int sq = unit / csplit, cs = unit - sq * csplit;
+  const int bi = sq / nb, bj = sq - bi * nb;
+  const bool busy = sq < nb * nb && bj >= bi;               // upper triangle of 4 x 4 blocks
+  double acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+  const int rot = threadIdx.x & 31;
+  for (int sub = 0; sub < kGramGroup; ++sub) {
+    const int chunk = grp * kGramGroup + sub;
+    if (chunk >= L.gchunks) break;
+    const int d0 = chunk * kGramCols;
+    __syncthreads();                                        // the previous chunk's values have been used
+    for (int i = threadIdx.x; i < r4 * kGramCols; i += 256) {
+      const int k = i / kGramCols, c = i - k * kGramCols;
+      const int d = d0 + c;
+      float y = 0.f;
+      if (k < r && d < L.d_in) {
+        for (int s = 0; s < L.slabs; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
+        L.Y[(long long)k * L.d_in + d] = y;
+      }
+      sY[i] = y;
     }
-    sY[i] = y;
+    __syncthreads();
+    if (busy) {
+      const float* yi = sY + (4 * bi) * kGramCols;
+      const float* yj = sY + (4 * bj) * kGramCols;
+      // rows are 128 floats apart, so all rows share a bank at equal c: every lane starts at its own
+      // column of its part (a fixed rotation, so the sum is the same on every run)
+      for (int c = 0; c < clen; ++c) {
+        const int cc = cs * clen + ((c + rot) & (clen - 1));
+        double a[4], b[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) { a[x] = (double)yi[x * kGramCols + cc]; b[x] = (double)yj[x * kGramCols + cc]; }
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+          for (int y = 0; y < 4; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
+      }
+    }
+  }
+  // the column parts of a block are added in a fixed order through shared memory
+  __syncthreads();
+  double* red = reinterpret_cast<double*>(gram_smem);     // [csplit][r4][r4]
+  if (busy) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) red[((size_t)cs * r4 + 4 * bi + x) * r4 + 4 * bj + y] = acc[x][y];
   }
   __syncthreads();
-  double* out = L.Gpart + (long long)chunk * r * r;
+  double* out = L.Gpart + (long long)grp * r * r;
   for (int p = threadIdx.x; p < r * r; p += 256) {
     const int i = p / r, j = p - i * r;
     if (j < i) continue;
-    double acc = 0.0;
-    const float* yi = sY + i * kGramCols;
-    const float* yj = sY + j * kGramCols;
-    // rows are 128 floats apart, so all rows share a bank at equal c: every lane starts at its own
-    // column (a fixed rotation, so the sum is still the same on every run)
-    const int rot = threadIdx.x & 31;
-    for (int c = 0; c < kGramCols; ++c) {
-      const int cc = (c + rot) & (kGramCols - 1);
-      acc = fma((double)yi[cc], (double)yj[cc], acc);
-    }
-    out[i * r + j] = acc;
+    double t = 0.0;
+    for (int q = 0; q < csplit; ++q) t += red[((size_t)q * r4 + i) * r4 + j];
+    out[p] = t;
   }
 }
 
@@ -212,7 +270,8 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
     const int i = p / r, j = p - i * r;
     double acc = 0.0;
     if (j >= i)
-      for (int c = 0; c < L.gchunks; ++c) acc += L.Gpart[(long long)c * r * r + p];   // fixed order
+      for (int c = 0; c < (L.gchunks + kGramGroup - 1) / kGramGroup; ++c)
+        acc += L.Gpart[(long long)c * r * r + p];   // fixed order
     S[i][j] = acc;
     Mm[p] = 0.0;
   }
@@ -256,29 +315,42 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
 }
 
 // ------------------------------------------------------------------ qr(Y), stage 3: Q = Y M
-// thread per column d; writes Q (fp32) into V and, for the tensor-core path, the bf16
-// hi/lo panels.
+// thread per column d, eight columns of Q at a time (M is upper triangular: column k needs Y's
+// columns 0..k); writes Q (fp32) into V and, for the tensor-core path, the bf16 hi/lo panels.
 __global__ void __launch_bounds__(128) apply_kernel(const DevLayer* __restrict__ layers, int l0) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const int d = blockIdx.x * 128 + threadIdx.x;
-  extern __shared__ __align__(16) double sM[];   // [r][r]
-  const int r = L.r;
-  for (int p = threadIdx.x; p < r * r; p += 128) sM[p] = L.M[p];
+  extern __shared__ __align__(16) double sM[];   // [r][r8], r8 = r rounded up to 8, padding zero
+  const int r = L.r, r8 = (r + 7) & ~7;
+  for (int p = threadIdx.x; p < r * r8; p += 128) {
+    const int j = p / r8, k = p - j * r8;
+    sM[p] = k < r ? L.M[j * r + k] : 0.0;
+  }
   __syncthreads();
   if (d >= L.d_in || blockIdx.x * 128 >= L.d_in) return;
-  float y[AGZO_MAX_RANK];
-#pragma unroll 4
-  for (int j = 0; j < r; ++j) y[j] = L.Y[(long long)j * L.d_in + d];
-  for (int k = 0; k < r; ++k) {
-    double acc = 0.0;
-    for (int j = 0; j <= k; ++j) acc = fma((double)y[j], sM[j * r + k], acc);
-    const float q = (float)acc;
-    L.V[(long long)k * L.ldv + d] = q;
-    if (L.Qb) {
-      const __nv_bfloat16 hi = __float2bfloat16_rn(q);
-      const __nv_bfloat16 lo = __float2bfloat16_rn(q - __bfloat162float(hi));
-      L.Qb[(long long)k * L.d_in + d] = hi;
-      L.Qb[(long long)(L.NP + k) * L.d_in + d] = lo;
+  for (int kb = 0; kb < r; kb += 8) {
+    double acc[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc[u] = 0.0;
+    const int jend = min(r, kb + 8);
+    for (int j = 0; j < jend; ++j) {
+      const double y = (double)L.Y[(long long)j * L.d_in + d];
+      const double* m = sM + j * r8 + kb;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc[u] = fma(y, m[u], acc[u]);   // M[j][k] = 0 for j > k
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int k = kb + u;
+      if (k >= r) break;
+      const float q = (float)acc[u];
+      L.V[(long long)k * L.ldv + d] = q;
+      if (L.Qb) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(q);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(q - __bfloat162float(hi));
+        L.Qb[(long long)k * L.d_in + d] = hi;
+        L.Qb[(long long)(L.NP + k) * L.d_in + d] = lo;
+      }
     }
   }
   if (L.Qb) {   // padding rows of the operand panel stay zero
@@ -291,14 +363,14 @@ __global__ void __launch_bounds__(128) apply_kernel(const DevLayer* __restrict__
 
 cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s) {
   const int nl = w.l1 - w.l0;
-  reduce_gram_kernel<<<dim3(w.max_gchunks, nl), 256, (size_t)w.max_r * kGramCols * sizeof(float), s>>>(
+  reduce_gram_kernel<<<dim3((w.max_gchunks + kGramGroup - 1) / kGramGroup, nl), 256, gram_smem_bytes_upto(w.max_r), s>>>(
       w.d_layers, w.l0);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   chol_kernel<<<nl, kCholThreads, 0, s>>>(w.d_layers, w.l0, d_status);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  apply_kernel<<<dim3((w.max_din + 127) / 128, nl), 128, (size_t)w.max_r * w.max_r * sizeof(double), s>>>(
+  apply_kernel<<<dim3((w.max_din + 127) / 128, nl), 128, (size_t)w.max_r * ((w.max_r + 7) & ~7) * sizeof(double), s>>>(
       w.d_layers, w.l0);
   return cudaGetLastError();
 }
