@@ -36,6 +36,7 @@ struct Plan {
   std::vector<int> item_start;
   int total_items = 0;
   int max_rp = 0;
+  int max_b_bytes = 0;   // largest B operand area of a tensor-core pass item
   bool staged_r = false;           // the tensor-core pass copies R tiles that a fill kernel wrote to scratch
   int max_row_tiles = 0;
   size_t image_bytes = 0;
@@ -230,6 +231,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   plan->item_start.assign(n + 1, 0);
   plan->total_items = 0;
   plan->max_rp = 0;
+  plan->max_b_bytes = 0;
   const size_t base = kHeaderBytes + table_bytes(n);
   const size_t scratch_all = ws ? (ws_bytes > base ? ws_bytes - base : 0) : (size_t)-1;
   const size_t scratch_cap = ws ? scratch_all / regions / kAlign * kAlign : (size_t)-1;   // per region
@@ -289,6 +291,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       items += (long long)D.rtc_panels * D.rtc_chunks;
       if (items > 0x7fffffff) return AGZO_ERR_INVALID_ARG;
       if (D.rtc_rp > plan->max_rp) plan->max_rp = D.rtc_rp;
+      plan->max_b_bytes = std::max(plan->max_b_bytes, rmw_tc_b_bytes(D));
       if (ws) D.wmap = ws + maps_offset(n) + (size_t)i * kMapBytes + 384;
     } else if (a.W) {
       if (vec) plan->fast_mode_mask |= 1 << D.rmw_mode; else plan->any_slow = true;
@@ -481,7 +484,7 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   if (st != AGZO_OK) return st;
   if (c->plan.total_items > 0) {
     Timed t(c, AGZO_KC_RMW_TC, s, c->plan.staged_r ? 2 : 1);
-    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->plan.max_row_tiles, c->plan.staged_r,
+    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->plan.max_r, c->plan.max_b_bytes, c->plan.max_row_tiles, c->plan.staged_r,
                         c->rmw_tc_slots, c->rmw_tc_inflight, seed,
                         coef, d_coef, dev_status(c), c->sm_count, s));
   }

@@ -54,7 +54,7 @@ struct alignas(16) DevLayer {
   int rtc_np;            // column panels per item (they share the R operand of a row tile)
   int rtc_chunk_blocks;  // 128-row blocks per row chunk
   int rtc_cw;            // columns per panel: 256, 128 or 64
-  int rtc_rp;            // rank rounded up to a multiple of 8
+  int rtc_rp;            // rank rounded up to a multiple of 16
   // staged R: for r > 16 the split A operand of every 128-row tile is written once per pass to
   // scratch, in the exact shared-memory layout, and the pass copies it in instead of regenerating
   // it for every column panel.  rimg = this layer's first tile image, null = regenerate in the kernel

@@ -7,9 +7,11 @@
 // (M = 128, N = the panel's columns, K = 4 * rp), its fp32 result waits in TMEM, and the only
 // per-weight work left for the CUDA cores is  w + c * delta  and the rounding to bf16.
 //
-// Precision: R and A^T are fp32; each is split as hi + lo in bf16 and the four cross products
-// are laid side by side along K (K index = [RhAh | RhAl | RlAh | RlAl]), so the products are
-// exact and summed in fp32; what is dropped is below 2^-17 of each term.
+// Precision: R and A^T are fp32; each is split as hi + lo in bf16.  The operands hold each part
+// once (A operand = [Rh | Rl], B operand = [Ah | Al], rp columns each) and the chain runs over
+// the four cross products Rh Ah, Rh Al, Rl Ah, Rl Al by pointing the instruction descriptors at
+// the parts, so the products are exact and summed in fp32; what is dropped is below 2^-17 of
+// each term.
 //
 // Work item = (layer, chunk of up to 8 row tiles, group of up to two adjacent column panels).
 // The R operand of a row tile serves every panel of the group, so R is regenerated once per
@@ -48,6 +50,11 @@ constexpr int kWarpLoader = 0, kWarpMma = 1, kWarpStorer = 2, kWarpEpi0 = 3, kNu
               kWarpGen0 = kWarpEpi0 + kNumEpiWarps, kMaxGenWarps = 8;
 constexpr int kMaxThreads = (kWarpGen0 + kMaxGenWarps) * 32;   // 608
 constexpr uint32_t kTmemCols = 512;        // two delta buffers of up to 256 columns
+
+// rp = the rank rounded up to a multiple of 16 (one instruction takes K = 16); an operand row is
+// 2 * rp bf16 values, stored as K atoms of 64
+__host__ __device__ inline int rtc_rank_padded(int r) { return (r + 15) & ~15; }
+__host__ __device__ inline int rtc_katoms(int rp) { return (2 * rp + 63) / 64; }
 
 struct Shared {
   uint64_t full_w[kMaxSlots];    // TMA load of the slot landed
@@ -115,16 +122,14 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4* hi, uint4* lo
   lo->z = pack2(lo_part(v[4]), lo_part(v[5])); lo->w = pack2(lo_part(v[6]), lo_part(v[7]));
 }
 
-// Writes group g (8 consecutive rank indices) of one operand row: the hi part goes to K terms
-// t0a and t0b, the lo part to t1a and t1b (term t occupies K indices [t*rp, (t+1)*rp)).
-__device__ __forceinline__ void put_group(uint8_t* base, int atom_bytes, int row, int g, int g8, uint4 hi, uint4 lo,
-                                          int t_hi_a, int t_hi_b, int t_lo_a, int t_lo_b) {
-  const int terms[4] = {t_hi_a, t_hi_b, t_lo_a, t_lo_b};
+// Writes group g (8 consecutive rank indices) of one operand row: the hi parts at K index 8g,
+// the lo parts at rp + 8g (g8 = rp / 8 groups per part).
+__device__ __forceinline__ void put_group(uint8_t* base, int atom_bytes, int row, int g, int g8, uint4 hi, uint4 lo) {
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int cg = terms[q] * g8 + g;              // 16-byte chunk index along K
+  for (int q = 0; q < 2; ++q) {
+    const int cg = q * g8 + g;                     // 16-byte chunk index along K
     uint8_t* p = base + (cg >> 3) * atom_bytes + swz(row, cg & 7);
-    *reinterpret_cast<uint4*>(p) = q < 2 ? hi : lo;
+    *reinterpret_cast<uint4*>(p) = q == 0 ? hi : lo;
   }
 }
 
@@ -163,14 +168,15 @@ __device__ __forceinline__ void gen_r_group(const DevLayer& L, long long row, in
 
 __global__ void __launch_bounds__(kMaxThreads, 1)
 rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_start, int n_layers,
-              int total_items, int a_bufs, int a_buf_bytes, int slots, int inflight, int staged, uint64_t seed,
+              int total_items, int a_bufs, int a_buf_bytes, int b_area_bytes, int slots, int inflight, int staged,
+              uint64_t seed,
               float coef_imm,
               const float* __restrict__ d_coef, DevStatus* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = base;                                   // a_bufs x a_buf_bytes
-  uint8_t* sB = sA + (size_t)a_bufs * a_buf_bytes;      // kMaxPanels x kBBytes
-  uint8_t* sW = sB + kMaxPanels * kBBytes;              // slots x kBoxBytes
+  uint8_t* sB = sA + (size_t)a_bufs * a_buf_bytes;      // two panels of kBBytes, or one larger panel
+  uint8_t* sW = sB + b_area_bytes;                      // slots x kBoxBytes
   __shared__ Shared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gen_warps = (int)(blockDim.x >> 5) - kWarpGen0;   // 4 for small ranks, 8 otherwise
@@ -264,7 +270,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
         const Item it = decode_item(layers, item_start, n_layers, item);
         if (!mbar_wait(&sh.b_full, ic & 1)) { ok = false; break; }
         const uint32_t idesc = instr_desc(kRows, it.cw, 0, 0);
-        const int ksteps = it.rp / 4;                    // K = 4 * rp, 16 per instruction
+        const int kpt = it.rp >> 4;                      // instructions (K = 16) per cross product
         const uint32_t b_atom = (uint32_t)it.cw * 128u;
         for (int rb = it.rb0; rb < it.rb1 && ok; ++rb, ++ta) {
           const int ab = ta % a_bufs, au = ta / a_bufs;
@@ -275,11 +281,14 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
             if (tu > 0 && !mbar_wait(&sh.tmem_empty[tb], (tu - 1) & 1)) { ok = false; break; }
             tc_fence_after();
             const uint32_t b0 = smem_u32(sB + (size_t)p * kBBytes);
-            for (int ks = 0; ks < ksteps; ++ks) {
-              const int ka = ks >> 2, kk = ks & 3;
-              const uint64_t ad = smem_desc(a0 + ka * kAtomBytesA + kk * 32, 0, 1024);
-              const uint64_t bd = smem_desc(b0 + ka * b_atom + kk * 32, 0, 1024);
-              mma_bf16(tmem + (uint32_t)tb * 256u, ad, bd, idesc, ks > 0 ? 1u : 0u);
+            for (int term = 0; term < 4; ++term) {       // Rh Ah, Rh Al, Rl Ah, Rl Al
+              const int ka0 = (term & 2) ? it.rp : 0, kb0 = (term & 1) ? it.rp : 0;   // first K index of the part
+              for (int j = 0; j < kpt; ++j) {
+                const int ka = ka0 + 16 * j, kb = kb0 + 16 * j;
+                const uint64_t ad = smem_desc(a0 + (ka >> 6) * kAtomBytesA + (ka & 63) * 2, 0, 1024);
+                const uint64_t bd = smem_desc(b0 + (kb >> 6) * b_atom + (kb & 63) * 2, 0, 1024);
+                mma_bf16(tmem + (uint32_t)tb * 256u, ad, bd, idesc, (term | j) ? 1u : 0u);
+              }
             }
             mma_commit(&sh.tmem_full[tb]);
           }
@@ -301,7 +310,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
       const Item it = decode_item(layers, item_start, n_layers, item);
       const DevLayer& L = *it.L;
       const int r = L.r, g8 = it.rp >> 3;
-      // B operand: row n = column col0 + n of the panel, K = [Ah | Al | Ah | Al]
+      // B operand: row n = column col0 + n of the panel, K = [Ah | Al]
       if (ic > 0) {
         ok = mbar_wait(&sh.b_empty, (ic - 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
@@ -321,12 +330,15 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
         }
         uint4 hi, lo;
         split8(v, &hi, &lo);
-        put_group(sB + (size_t)p * kBBytes, b_atom, n, g, g8, hi, lo, 0, 2, 1, 3);
+        put_group(sB + (size_t)p * kBBytes, b_atom, n, g, g8, hi, lo);
       }
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.b_full);
-      // A operand per tile: row i = R[rb*128 + i][:], K = [Rh | Rh | Rl | Rl]
+      // A operand per tile: row i = R[rb*128 + i][:], K = [Rh | Rl]
+      // Staged R needs one thread per tile.  Only its warp walks the tiles: a warp that waited on
+      // a_empty without feeding a_full could fall two phases behind and take a later phase for its own.
+      if (staged && warp != kWarpGen0) continue;
       for (int rb = it.rb0; rb < it.rb1; ++rb, ++t) {
         const int ab = t % a_bufs, au = t / a_bufs;
         if (au > 0) {
@@ -347,7 +359,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
           const int g = unit >> 7, i = unit & (kRows - 1);
           uint4 hi, lo;
           gen_r_group(L, (long long)rb * kRows + i, g, seed, &hi, &lo);
-          put_group(a_base, kAtomBytesA, i, g, g8, hi, lo, 0, 1, 2, 3);
+          put_group(a_base, kAtomBytesA, i, g, g8, hi, lo);
         }
         fence_proxy_async();
         __syncwarp();
@@ -421,7 +433,7 @@ rmw_tc_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ item_
   if (warp == kWarpMma) { tc_fence_after(); tmem_dealloc(tmem, kTmemCols); }
 }
 
-// Staged R: CTA = (row tile, layer); writes the tile's split A operand [Rh | Rh | Rl | Rl] to
+// Staged R: CTA = (row tile, layer); writes the tile's split A operand [Rh | Rl] to
 // scratch exactly as rmw_tc_kernel lays it out in shared memory (K atoms of [128 rows][128 bytes],
 // 128-byte swizzle), so the pass can bulk-copy it.
 __global__ void __launch_bounds__(256) rmw_tc_fill_r_kernel(const DevLayer* __restrict__ layers, uint64_t seed) {
@@ -435,7 +447,7 @@ __global__ void __launch_bounds__(256) rmw_tc_fill_r_kernel(const DevLayer* __re
     const int g = unit >> 7, i = unit & (kRows - 1);
     uint4 hi, lo;
     gen_r_group(L, (long long)rb * kRows + i, g, seed, &hi, &lo);
-    put_group(img, kAtomBytesA, i, g, g8, hi, lo, 0, 1, 2, 3);
+    put_group(img, kAtomBytesA, i, g, g8, hi, lo);
   }
 }
 
@@ -448,24 +460,24 @@ bool rmw_tc_eligible(const agzo_layer& a) {
 }
 
 void rmw_tc_shape(const agzo_layer& a, int panels, bool staged, DevLayer* D) {
-  const int rp = (a.r + 7) & ~7;
-  const int katoms = (4 * rp + 63) / 64;                 // 1, 2, 3 or 4 K atoms of 64
-  // Panel width: K atoms x columns x 128 bytes of B operand must fit its area (32 KiB per panel,
-  // 64 KiB when one panel takes both).  With R staged in scratch there is nothing to amortise over
-  // a second panel, so one wide panel is used (fewer, larger MMAs).
-  const int cw = katoms == 1 ? 256 : staged ? (katoms == 2 ? 256 : 128) : (katoms == 2 ? 128 : 64);
-  // panels == 0: one panel per item while R is cheap to regenerate (rp <= 16: the pass is
+  const int rp = rtc_rank_padded(a.r);
+  const int katoms = rtc_katoms(rp);                     // 1 (rp <= 32) or 2 K atoms of 64
+  // panels == 0: one panel per item while R is cheap to regenerate (rp = 16: the pass is
   // HBM-bound either way and the smaller items balance better), two from there on, where
-  // regenerating R is what limits the pass
-  int np = panels == 1 ? 1 : panels == 2 ? kMaxPanels : (katoms == 1 ? 1 : kMaxPanels);
-  if (staged && katoms >= 2) np = 1;
+  // regenerating R is what limits the pass.  With R staged in scratch there is nothing to
+  // amortise over a second panel.
+  int np = panels == 1 ? 1 : panels == 2 ? kMaxPanels : (rp <= 16 ? 1 : kMaxPanels);
+  if (staged && rp > 16) np = 1;
+  // Panel width: K atoms x columns x 128 bytes of B operand; a panel of a pair has 32 KiB, a
+  // single panel may take 64 KiB
+  const int cw = (katoms == 1 || np == 1) ? 256 : 128;
   D->rtc_rp = rp;
   D->rtc_cw = cw;
   D->rtc_np = np;
   D->rtc_panels = (a.d_in + np * cw - 1) / (np * cw);   // panel groups
   // row tiles per item: the B operand is rebuilt once per item, which stalls the MMA pipeline for a
   // few microseconds when the rank is large, so those items are taller
-  D->rtc_chunk_blocks = katoms >= 2 ? 32 : 8;
+  D->rtc_chunk_blocks = rp >= 32 ? 32 : 8;
   const int nrb = (a.d_out + kRows - 1) / kRows;
   D->rtc_chunks = (nrb + D->rtc_chunk_blocks - 1) / D->rtc_chunk_blocks;
 }
@@ -480,14 +492,19 @@ cudaError_t rmw_tc_init() {
   return cudaFuncSetAttribute(rmw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
 }
 
+int rmw_tc_b_bytes(const DevLayer& D) {
+  return D.rtc_np > 1 ? kMaxPanels * kBBytes : D.rtc_cw * rtc_katoms(D.rtc_rp) * 128;
+}
+
 size_t rmw_tc_image_bytes(const agzo_layer& a) {
-  const int rp = (a.r + 7) & ~7;
-  const size_t katoms = (size_t)(4 * rp + 63) / 64;
+  const int rp = rtc_rank_padded(a.r);
+  const size_t katoms = (size_t)rtc_katoms(rp);
   return (size_t)((a.d_out + kRows - 1) / kRows) * katoms * kAtomBytesA;
 }
 
 cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
-                          int max_rp, int max_row_tiles, bool staged, int slots_wanted, int inflight, uint64_t seed,
+                          int max_rp, int max_r, int max_b_bytes, int max_row_tiles, bool staged, int slots_wanted, int inflight,
+                          uint64_t seed,
                           float coef, const float* d_coef, DevStatus* d_status, int sm_count, cudaStream_t s) {
   if (total_items <= 0) return cudaSuccess;
   if (staged) {
@@ -495,25 +512,23 @@ cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  const int katoms = (4 * max_rp + 63) / 64;
+  const int katoms = rtc_katoms(max_rp);
   const int a_buf_bytes = katoms * kAtomBytesA;
-  // one A buffer where two would leave too few ring slots; with staged R the buffer is refilled by a
-  // bulk copy that is short next to the tile's HBM time
-  const int a_bufs = (katoms >= 3 || (staged && katoms >= 2)) ? 1 : 2;
-  const int fixed = a_bufs * a_buf_bytes + kMaxPanels * kBBytes;
+  const int a_bufs = 2;                       // one being refilled while the other feeds the chain
+  const int fixed = a_bufs * a_buf_bytes + max_b_bytes;
   int slots = (224 * 1024 - fixed) / kBoxBytes;
   if (slots > kMaxSlots) slots = kMaxSlots;
   if (slots_wanted >= 2 && slots_wanted < slots) slots = slots_wanted;
   const size_t smem = (size_t)fixed + (size_t)slots * kBoxBytes + 1024;
   const int grid = total_items < sm_count ? total_items : sm_count;
-  // operand-builder warps: four keep up with the stream for rp = 8, larger ranks get eight
-  const int threads = (kWarpGen0 + (max_rp <= 8 ? 4 : kMaxGenWarps)) * 32;
+  // operand-builder warps: four keep up with the stream for r <= 8, larger ranks get eight
+  const int threads = (kWarpGen0 + (max_r <= 8 ? 4 : kMaxGenWarps)) * 32;
   // loads in flight per CTA: enough to cover the HBM latency at this SM's share of the
   // bandwidth (4 to 5 boxes of 16 KiB); more only lengthens the queues in front of the stores
-  if (inflight < 1) inflight = max_rp <= 8 ? 4 : 5;
+  if (inflight < 1) inflight = max_r <= 8 ? 4 : 5;
   if (inflight > slots) inflight = slots;
   rmw_tc_kernel<<<grid, threads, smem, s>>>(d_layers, d_item_start, n_layers, total_items, a_bufs, a_buf_bytes,
-                                             slots, inflight, staged ? 1 : 0, seed, coef, d_coef, d_status);
+                                             max_b_bytes, slots, inflight, staged ? 1 : 0, seed, coef, d_coef, d_status);
   return cudaGetLastError();
 }
 
