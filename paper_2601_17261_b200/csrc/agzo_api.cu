@@ -171,12 +171,15 @@ bool same_input(const agzo_layer& a, const agzo_layer& b) {
 }
 
 // Token slabs of the X^T T product.  CUDA-core kernels: 32 slabs at most.  Tensor-core
-// kernels: slabs of 2048 tokens (32 pipeline steps per CTA) when the layer has that many; a
-// wave holds many layers, so the grid is filled by the layers, not by thin slabs.
-void slab_shape(const agzo_layer& a, bool tc, int* slabs, int* slab_rows) {
+// kernels: slabs of 2048 tokens (32 pipeline steps per CTA) when the layer has that many.  When
+// the call's layers fill the grid by their column blocks alone (long_slabs), a slab is up to
+// 16384 tokens: every slab costs a partial Y (r x d_in floats written, and read again by the
+// panel QR), and the CTAs' pipelines start and drain less often.
+constexpr int kLongSlabColumnBlocks = 1024;   // 128-column blocks over all layers from which slabs are long
+void slab_shape(const agzo_layer& a, bool tc, bool long_slabs, int* slabs, int* slab_rows) {
   int rows;
   if (tc) {
-    rows = a.m >= 8192 ? 2048 : (a.m + 3) / 4;
+    rows = a.m >= 8192 ? (long_slabs ? (a.m < 16384 ? a.m : 16384) : 2048) : (a.m + 3) / 4;
     rows = (rows + 63) / 64 * 64;
   } else {
     rows = (a.m + 31) / 32;
@@ -188,10 +191,10 @@ void slab_shape(const agzo_layer& a, bool tc, int* slabs, int* slab_rows) {
 }
 
 // scratch bytes one layer needs for extraction (0 when it has no X)
-size_t layer_scratch(const agzo_layer& a, bool tc, bool with_panels = true) {
+size_t layer_scratch(const agzo_layer& a, bool tc, bool long_slabs, bool with_panels = true) {
   if (!has_x(a)) return 0;
   int slabs, slab_rows;
-  slab_shape(a, tc, &slabs, &slab_rows);
+  slab_shape(a, tc, long_slabs, &slabs, &slab_rows);
   const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
   const size_t gch = (d + 127) / 128;
   size_t b = 0;
@@ -312,6 +315,10 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
 
   // extraction waves: consecutive layers whose activations fit the wave budget and whose
   // scratch fits the workspace
+  long long column_blocks = 0;
+  for (int k = 0; k < n; ++k)
+    if (has_x(L[k]) && extract_path != 1 && tc_available && tc_eligible(L[k])) column_blocks += (L[k].d_in + 127) / 128;
+  const bool long_slabs = column_blocks >= kLongSlabColumnBlocks && !opts.extract_fused;
   int i = 0;
   while (i < n) {
     if (!has_x(L[i])) { ++i; plan->wave_end.push_back(i); plan->wave_region.push_back(-1); continue; }
@@ -335,7 +342,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       }
       auto unit_need = [&](int len, int nrows) {
         size_t b = 0;
-        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, false);
+        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, long_slabs, false);
         if (tc) b += tc_panel_bytes(L[j], nrows);
         return b;
       };
@@ -355,7 +362,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
           DevLayer& D = plan->dev[j + g];
           const agzo_layer& a = L[j + g];
           int slabs, slab_rows;
-          slab_shape(a, tc, &slabs, &slab_rows);
+          slab_shape(a, tc, long_slabs, &slabs, &slab_rows);
           const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
           const size_t gch = (d + 127) / 128;
           D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
