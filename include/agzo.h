@@ -129,7 +129,7 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),
  * "rmw_tc_panels" (column panels per work item, 1 or 2); "rmw_stage_r" 0 = when some layer's rank
  * exceeds 16 the split R operand of every 128-row tile is written once per pass to the scratch
- * area (d_out x 8 r' bytes per layer, r' = r rounded up to 8) and copied in by the pass instead of
+ * area (d_out x 4 r' bytes per layer, r' = r rounded up to 16) and copied in by the pass instead of
  * being regenerated for every column panel, 1 = never, 2 = always;
  * "share_inputs" 1 (default) = consecutive layers whose X is the same buffer (same pointer, pitch,
  * m, d_in: q/k/v or gate/up of a transformer block) are served by one sweep over X per product,
@@ -143,6 +143,31 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * "time_kernel_class" = one agzo_kernel_class whose launches get a CUDA event pair on the
  * caller's stream (0 = none), read back by agzo_read_counters.                           */
 agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value);
+
+/* Token-sharded extraction over data-parallel ranks.  Algorithm 1 touches the activations only
+ * through the products H Omega = X^T Omega, H^T Q = X Q and H T = X^T T, and the tokens (the
+ * columns of H, m = batch x sequence of them) enter the last one as a sum: with the batch split
+ * over ranks, rank p holding the rows X_p of X from global token `token_offset` on,
+ *     Y = X^T T = sum_p X_p^T (X_p Q),
+ * so every rank computes its own term and the Y panels are summed over the ranks before each
+ * qr(Y).  All ranks then hold the same Y, hence the same V, bit for bit.  The paper runs on one
+ * device and has no counterpart of this call.
+ *
+ * fn: called on the host, K + 1 times per wave of layers, after the launches that produce the
+ * wave's Y panels have been enqueued on `stream`.  `d_buf` is ONE contiguous device buffer of
+ * `count` floats that holds all those panels (and alignment gaps, whose content is arbitrary);
+ * fn must enqueue on `stream` an in-place sum of it over all ranks (an all-reduce, e.g.
+ * ncclAllReduce(d_buf, d_buf, count, ncclFloat, ncclSum, comm, stream)) and return 0; a non-zero
+ * return ends the call with AGZO_ERR_CALLBACK.  Every rank must pass the same layers (same
+ * d_in, r, layer_id; m may differ), the same seed, K and options, so that the ranks make the
+ * same sequence of calls with the same counts.
+ * token_offset: global index of this rank's first token; row t of the local X is row
+ * token_offset + t of the batch and draws that row of the Gaussian test matrix Omega.
+ * fn = NULL (with token_offset 0) returns to single-rank extraction.  While fn is set, waves run
+ * one after another on the caller's stream ("extract_streams" is taken as 1).
+ * The buffer is owned by the library (it lies in the workspace); fn must not keep the pointer. */
+typedef int (*agzo_allreduce_fn)(void* user, void* stream, float* d_buf, size_t count);
+agzo_status agzo_set_allreduce(agzo_ctx* ctx, agzo_allreduce_fn fn, void* user, int64_t token_offset);
 
 typedef enum agzo_kernel_class {
   AGZO_KC_NONE = 0,

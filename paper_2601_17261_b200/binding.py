@@ -31,7 +31,7 @@ EXPORTS = [
     "agzo_status_string", "agzo_last_cuda_error", "agzo_extract_subspace", "agzo_perturb",
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
-    "agzo_extract_subspace_static", "agzo_fill_gaussian_basis",
+    "agzo_extract_subspace_static", "agzo_fill_gaussian_basis", "agzo_set_allreduce",
 ]
 KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC, KC_FUSED_POWER = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
@@ -55,6 +55,7 @@ class agzo_params(C.Structure):
 
 
 LOSS_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p)
+ALLREDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t)
 
 _lib = None
 
@@ -97,6 +98,7 @@ def lib() -> C.CDLL:
         "agzo_debug_philox": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_debug_gaussian": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_read_counters": (i32, [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)]),
+        "agzo_set_allreduce": (i32, [vp, ALLREDUCE_FN, vp, i64]),
         "agzo_extract_subspace_static": (i32, [vp, i64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                C.c_int32, u64, u32, vp, i64, vp, vp]),
     }
@@ -310,6 +312,58 @@ def agzo_step(ctx: Context, layers, *, seed: int, eps: float, lr: float, K: int,
     if st == AGZO_ERR_CALLBACK and err:
         raise AgzoError(st, f"agzo_step (callback raised {err[0]!r})")
     _check(st, "agzo_step")
+
+
+class _DeviceFloats:
+    """A float32 device buffer given by address, for torch.as_tensor (no copy)."""
+
+    def __init__(self, ptr: int, count: int):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": "<f4", "data": (ptr, False),
+                                         "version": 2}
+
+
+def device_floats(ptr: int, count: int, device: int) -> torch.Tensor:
+    """View of `count` floats at device address `ptr` (memory owned by someone else)."""
+    return torch.as_tensor(_DeviceFloats(ptr, count), device=f"cuda:{device}")
+
+
+def agzo_set_allreduce(ctx: Context, fn, token_offset: int = 0) -> None:
+    """fn(buf: torch.Tensor, stream_ptr: int) -> None sums the float32 device view `buf` over
+    all ranks in place, enqueued on the stream; None (with token_offset 0) switches
+    token-sharded extraction off.  The context keeps the callback alive."""
+    if fn is None:
+        _check(lib().agzo_set_allreduce(ctx.handle, ALLREDUCE_FN(), None, 0), "agzo_set_allreduce")
+        ctx._allreduce_cb = None
+        return
+    errors: List[BaseException] = []
+
+    def tramp(user, stream_ptr, d_buf, count):
+        try:
+            fn(device_floats(int(d_buf), int(count), ctx.device), int(stream_ptr or 0))
+            return 0
+        except BaseException as e:  # noqa: BLE001 - must not unwind through C
+            errors.append(e)
+            return 1
+
+    cb = ALLREDUCE_FN(tramp)
+    _check(lib().agzo_set_allreduce(ctx.handle, cb, None, int(token_offset)), "agzo_set_allreduce")
+    ctx._allreduce_cb = cb
+    ctx._allreduce_errors = errors
+
+
+def torch_allreduce(group=None):
+    """An `fn` for agzo_set_allreduce that sums with torch.distributed (NCCL for device
+    buffers) on the stream the library passes."""
+    import torch.distributed as dist
+
+    def fn(buf: torch.Tensor, stream_ptr: int) -> None:
+        if buf.is_cuda:
+            with torch.cuda.stream(torch.cuda.ExternalStream(stream_ptr, device=buf.device)):
+                dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+        else:
+            dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+
+    return fn
 
 
 def agzo_perturb_dense(ctx: Context, w: torch.Tensor, seed: int, layer_id: int, scale: float,

@@ -26,6 +26,10 @@ struct Plan {
   std::vector<int> tile_start;     // n + 1
   std::vector<int> wave_end;       // exclusive end index of each extraction wave
   std::vector<int> wave_region;    // scratch region (= helper stream) of each wave, -1 = nothing to do
+  // the Y panels of a wave's layers lie one after another at the end of the wave's scratch, so that a
+  // token-sharded run can sum all of them over the ranks in one call
+  std::vector<float*> wave_y;
+  std::vector<size_t> wave_y_count;   // floats, alignment gaps included
   int regions = 1;
   int total_tiles = 0;
   int max_r = 0;
@@ -76,6 +80,9 @@ struct agzo_ctx {
   int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
   int extract_fused;       // 1: fused power-step kernel where a layer's shape allows it
   int share_inputs;        // 1: consecutive layers with the same X share the sweeps over it
+  agzo_allreduce_fn allreduce;   // token-sharded extraction: sums a wave's Y panels over the ranks
+  void* allreduce_user;
+  int64_t token_offset;    // global index of this rank's first token
   cudaStream_t aux[2];     // helper streams of extraction, forked from and joined to the caller's stream
   cudaEvent_t fork_ev, join_ev[2];
   // descriptors last uploaded
@@ -225,6 +232,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   plan->tile_start.assign(n + 1, 0);
   plan->wave_end.clear();
   plan->wave_region.clear();
+  plan->wave_y.clear();
+  plan->wave_y_count.clear();
   const int regions = opts.extract_regions == 2 ? 2 : 1;
   plan->regions = regions;
   plan->max_r = 0;
@@ -321,10 +330,15 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   const bool long_slabs = column_blocks >= kLongSlabColumnBlocks && !opts.extract_fused;
   int i = 0;
   while (i < n) {
-    if (!has_x(L[i])) { ++i; plan->wave_end.push_back(i); plan->wave_region.push_back(-1); continue; }
+    if (!has_x(L[i])) {
+      ++i;
+      plan->wave_end.push_back(i); plan->wave_region.push_back(-1);
+      plan->wave_y.push_back(nullptr); plan->wave_y_count.push_back(0);
+      continue;
+    }
     const int region = real_waves++ % regions;
     plan->has_extract = true;
-    size_t used = 0;
+    size_t used = 0, used_y = 0;    // scratch of the wave so far; the part of it that is Y panels
     int64_t xbytes = 0;
     int j = i;
     const bool wave_tc = extract_path != 1 && tc_available && tc_eligible(L[i]);
@@ -356,8 +370,10 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       }
       if (used + need > scratch_cap) return AGZO_ERR_WORKSPACE;
       // carve
+      size_t need_y = 0;
+      for (int g = 0; g < glen; ++g) need_y += align_up((size_t)L[j + g].r * (size_t)L[j + g].d_in * 4);
       if (ws) {
-        char* p = ws + base + (size_t)region * scratch_cap + used;
+        char* p = ws + base + (size_t)region * scratch_cap + (used - used_y);
         for (int g = 0; g < glen; ++g) {
           DevLayer& D = plan->dev[j + g];
           const agzo_layer& a = L[j + g];
@@ -368,7 +384,6 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
           D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
           D.T = reinterpret_cast<float*>(p);      p += align_up(m * r * 4);
           D.Ypart = reinterpret_cast<float*>(p);  p += align_up((size_t)slabs * r * d * 4);
-          D.Y = reinterpret_cast<float*>(p);      p += align_up(r * d * 4);
           D.Gpart = reinterpret_cast<double*>(p); p += align_up(gch * r * r * 8);
           D.M = reinterpret_cast<double*>(p);     p += align_up(r * r * 8);
         }
@@ -389,10 +404,21 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
         }
       }
       used += need;
+      used_y += need_y;
       xbytes += xb;
       j += glen;
     }
     if (used > max_wave_scratch) max_wave_scratch = used;
+    {   // the Y panels follow everything else of the wave
+      char* y0 = ws ? ws + base + (size_t)region * scratch_cap + (used - used_y) : nullptr;
+      char* y = y0;
+      for (int k = i; k < j && ws; ++k) {
+        plan->dev[k].Y = reinterpret_cast<float*>(y);
+        y += align_up((size_t)L[k].r * (size_t)L[k].d_in * 4);
+      }
+      plan->wave_y.push_back(reinterpret_cast<float*>(y0));
+      plan->wave_y_count.push_back(used_y / 4);
+    }
     {   // order in which T = X Q takes the wave's layers: largest d_in first (stable)
       std::vector<int> ord(j - i);
       for (int k = 0; k < j - i; ++k) ord[k] = k;
@@ -429,7 +455,8 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
   PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels, c->rmw_stage_r,
-                c->tc.available, c->extract_fused != 0, c->share_inputs != 0, c->extract_streams};
+                c->tc.available, c->extract_fused != 0, c->share_inputs != 0,
+                c->allreduce ? 1 : c->extract_streams};   // the ranks' sums run in wave order on the caller's stream
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
     opts.extract_regions = 1;
@@ -569,6 +596,9 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->wave_bytes = kDefaultWaveBytes;
   c->extract_streams = 2;
   c->extract_fused = 0;
+  c->allreduce = nullptr;
+  c->allreduce_user = nullptr;
+  c->token_offset = 0;
   c->share_inputs = 1;
   c->aux[0] = c->aux[1] = nullptr;
   c->fork_ev = c->join_ev[0] = c->join_ev[1] = nullptr;
@@ -671,6 +701,16 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
   return AGZO_OK;
 }
 
+agzo_status agzo_set_allreduce(agzo_ctx* ctx, agzo_allreduce_fn fn, void* user, int64_t token_offset) {
+  if (!ctx || ctx->magic != kMagic) return AGZO_ERR_STATE;
+  if (token_offset < 0 || (!fn && token_offset != 0)) return AGZO_ERR_INVALID_ARG;
+  ctx->allreduce = fn;
+  ctx->allreduce_user = user;
+  ctx->token_offset = token_offset;
+  ctx->cached_valid = false;   // the number of scratch regions depends on it
+  return AGZO_OK;
+}
+
 agzo_status agzo_read_counters(agzo_ctx* ctx, double* h_ms, int64_t* h_timed, int64_t* h_total) {
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
@@ -735,6 +775,8 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
       ExtractWave w{};
       w.d_layers = dev_layers(ctx);
       w.l0 = l0; w.l1 = l1;
+      w.omega_row0 = ctx->allreduce ? ctx->token_offset : 0;
+      w.y_reduced = ctx->allreduce ? 1 : 0;
       bool all_tc = ctx->extract_path != 1;
       for (int i = l0; i < l1; ++i) {
         const DevLayer& D = P.dev[i];
@@ -752,6 +794,16 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
       auto panel_qr = [&]() -> cudaError_t {
         Timed t(ctx, AGZO_KC_PANEL_QR, ws, 3);
         return launch_panel_qr(w, dst, ws);
+      };
+      // token-sharded run: Y = sum over ranks of X_p^T T_p, all panels of the wave in one call
+      auto sum_over_ranks = [&]() -> agzo_status {
+        if (!ctx->allreduce) return AGZO_OK;
+        {
+          Timed t(ctx, AGZO_KC_PANEL_QR, ws);
+          CU(ctx, launch_sum_slabs(w, ws));
+        }
+        if (ctx->allreduce(ctx->allreduce_user, ws, P.wave_y[wv], P.wave_y_count[wv]) != 0) return AGZO_ERR_CALLBACK;
+        return AGZO_OK;
       };
       auto omega = [&]() -> cudaError_t {
         Timed t(ctx, AGZO_KC_OMEGA, ws);
@@ -780,9 +832,11 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
         }
         return cudaSuccess;
       };
+      agzo_status sr;
       CU(ctx, omega());                        // Omega
       CU(ctx, xt_t(false));                    // Y <- H Omega
       for (int k = 0; k < K; ++k) {
+        if ((sr = sum_over_ranks()) != AGZO_OK) return sr;
         CU(ctx, panel_qr());                   // Q <- qr(Y)
         if (fz_classes) CU(ctx, power_fused());
         if (any_unfused) {
@@ -790,6 +844,7 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
           CU(ctx, xt_t(true));                 // Y <- H (H^T Q)
         }
       }
+      if ((sr = sum_over_ranks()) != AGZO_OK) return sr;
       CU(ctx, panel_qr());                     // A <- qr(Y)
     }
     return AGZO_OK;

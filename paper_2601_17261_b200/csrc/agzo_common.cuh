@@ -153,10 +153,13 @@ struct ExtractWave {
   const DevLayer* d_layers;   // device array (all layers)
   int l0, l1;
   int max_m, max_din, max_r, max_slabs, max_gchunks;
+  long long omega_row0;       // global index of the first local token (token-sharded extraction), else 0
+  int y_reduced;              // 1: Y already holds the sum over slabs (and ranks); the panel QR reads it as it is
 };
 cudaError_t launch_fill_omega(const ExtractWave& w, uint64_t seed, cudaStream_t s);
 cudaError_t launch_xt_t(const ExtractWave& w, cudaStream_t s);      // Ypart = X^T T per slab
 cudaError_t launch_x_q(const ExtractWave& w, cudaStream_t s);       // T = X Q (Q read from V)
+cudaError_t launch_sum_slabs(const ExtractWave& w, cudaStream_t s);   // Y = sum over slabs of Ypart
 cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s);
 
 }  // namespace agzo

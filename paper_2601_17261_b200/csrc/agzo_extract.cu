@@ -14,28 +14,31 @@
 namespace agzo {
 
 // ------------------------------------------------------------------ Omega -> T
-__global__ void fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed) {
+// Local token t is row row0 + t of the test matrix of the whole batch: element e of the stream is
+// (row0 + t) * r + k, so the Philox blocks that cover the local rows are walked, whatever row0 is.
+__global__ void fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed, long long row0) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const long long n = (long long)L.m * L.r;
-  const long long nb = (n + 3) >> 2;
-  for (long long b = blockIdx.x * (long long)blockDim.x + threadIdx.x; b < nb;
+  const long long e0 = row0 * L.r;
+  const long long b_end = (e0 + n + 3) >> 2;
+  for (long long b = (e0 >> 2) + blockIdx.x * (long long)blockDim.x + threadIdx.x; b < b_end;
        b += (long long)gridDim.x * blockDim.x) {
     const float4 g = gaussian_block((uint64_t)b, L.layer_id, kTagOmega, seed);
     const float gv[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
     for (int lane = 0; lane < 4; ++lane) {
-      const long long e = 4 * b + lane;
-      if (e < n) L.T[e] = gv[lane];
+      const long long e = 4 * b + lane - e0;
+      if (e >= 0 && e < n) L.T[e] = gv[lane];
     }
   }
 }
 
 cudaError_t launch_fill_omega(const ExtractWave& w, uint64_t seed, cudaStream_t s) {
-  const long long nb = ((long long)w.max_m * w.max_r + 3) >> 2;
+  const long long nb = (((long long)w.max_m * w.max_r + 3) >> 2) + 1;
   int gx = (int)((nb + 255) / 256);
   if (gx > 512) gx = 512;
   if (gx < 1) gx = 1;
-  fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed);
+  fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed, w.omega_row0);
   return cudaGetLastError();
 }
 
@@ -179,7 +182,7 @@ inline size_t gram_smem_bytes_upto(int max_r) {
   for (int r = 1; r <= max_r; ++r) b = gram_smem_bytes(r) > b ? gram_smem_bytes(r) : b;
   return b;
 }
-__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0) {
+__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0, int y_reduced) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const int ngroups = (L.gchunks + kGramGroup - 1) / kGramGroup;
   const int grp = blockIdx.x;
@@ -208,8 +211,12 @@ __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __rest
       const int d = d0 + c;
       float y = 0.f;
       if (k < r && d < L.d_in) {
-        for (int s = 0; s < L.slabs; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
-        L.Y[(long long)k * L.d_in + d] = y;
+        if (y_reduced) {
+          y = L.Y[(long long)k * L.d_in + d];
+        } else {
+          for (int s = 0; s < L.slabs; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
+          L.Y[(long long)k * L.d_in + d] = y;
+        }
       }
       sY[i] = y;
     }
@@ -361,10 +368,29 @@ __global__ void __launch_bounds__(128) apply_kernel(const DevLayer* __restrict__
   }
 }
 
+// Y[k][d] = sum_s Ypart[s][k][d] in slab order, on its own: token-sharded extraction sums Y over
+// the ranks before the panel QR reads it
+__global__ void __launch_bounds__(256) sum_slabs_kernel(const DevLayer* __restrict__ layers, int l0) {
+  const DevLayer& L = layers[l0 + blockIdx.y];
+  const long long n = (long long)L.r * L.d_in;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
+    float y = 0.f;
+    for (int s = 0; s < L.slabs; ++s) y += L.Ypart[(long long)s * n + i];
+    L.Y[i] = y;
+  }
+}
+
+cudaError_t launch_sum_slabs(const ExtractWave& w, cudaStream_t s) {
+  long long blocks = ((long long)w.max_r * w.max_din + 255) / 256;
+  if (blocks > 256) blocks = 256;
+  sum_slabs_kernel<<<dim3((unsigned)blocks, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s) {
   const int nl = w.l1 - w.l0;
   reduce_gram_kernel<<<dim3((w.max_gchunks + kGramGroup - 1) / kGramGroup, nl), 256, gram_smem_bytes_upto(w.max_r), s>>>(
-      w.d_layers, w.l0);
+      w.d_layers, w.l0, w.y_reduced);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   chol_kernel<<<nl, kCholThreads, 0, s>>>(w.d_layers, w.l0, d_status);

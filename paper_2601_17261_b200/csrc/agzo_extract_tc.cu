@@ -265,20 +265,22 @@ __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __r
 }
 
 // ---------------------------------------------------------------- Omega -> Tt (hi/lo), pads zero
-__global__ void tc_fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed) {
+// local token t is row row0 + t of the whole batch's test matrix (see fill_omega_kernel)
+__global__ void tc_fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed, long long row0) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const long long n = (long long)L.m * L.r;
-  const long long nb = (n + 3) >> 2;
+  const long long e0 = row0 * L.r;
+  const long long b_end = (e0 + n + 3) >> 2;
   const long long mp = L.m_pad;
   const int r = L.r, NP = L.NP;
-  for (long long b = blockIdx.x * (long long)blockDim.x + threadIdx.x; b < nb;
+  for (long long b = (e0 >> 2) + blockIdx.x * (long long)blockDim.x + threadIdx.x; b < b_end;
        b += (long long)gridDim.x * blockDim.x) {
     const float4 g = gaussian_block((uint64_t)b, L.layer_id, kTagOmega, seed);
     const float gv[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
     for (int lane = 0; lane < 4; ++lane) {
-      const long long e = 4 * b + lane;
-      if (e < n) {
+      const long long e = 4 * b + lane - e0;
+      if (e >= 0 && e < n) {
         const long long t = e / r;
         const int k = (int)(e - t * r);
         __nv_bfloat16 h, l;
@@ -413,11 +415,11 @@ bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps) {
 }
 
 cudaError_t tc_fill_omega(const TcState&, const ExtractWave& w, const DevLayer*, uint64_t seed, cudaStream_t s) {
-  const long long nb = ((long long)w.max_m * w.max_r + 3) >> 2;
+  const long long nb = (((long long)w.max_m * w.max_r + 3) >> 2) + 1;
   int gx = (int)((nb + 255) / 256);
   if (gx > 1024) gx = 1024;
   if (gx < 1) gx = 1;
-  tc_fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed);
+  tc_fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed, w.omega_row0);
   return cudaGetLastError();
 }
 
