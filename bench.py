@@ -220,6 +220,10 @@ def main():
                          "for a like-for-like step-overhead comparison")
     ap.add_argument("--blocks", type=int, default=0,
                     help="keep only the first N transformer blocks of the layer set (profiling-sized runs)")
+    ap.add_argument("--shard-tokens", action="store_true",
+                    help="every rank's activations are its own tokens of one batch of N x m tokens: extraction sums "
+                         "the Y panels over the ranks (NCCL all-reduce through agzo_set_allreduce); the in-place "
+                         "passes stay replicated.  Default: independent replicas")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -241,10 +245,12 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
-    if world > 1:
+    if world > 1 or args.shard_tokens:
         import torch.distributed as dist_mod
         dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29621")
+        dist.init_process_group("nccl", device_id=dev, rank=rank, world_size=world)
     B.lib()   # fails loudly when the CUDA library is missing
 
     Ws, Xs, Vs, layers = build_layer_set(cfg, r, dev, alias_inputs=args.alias_inputs)
@@ -262,6 +268,8 @@ def main():
     B.agzo_set_option(ctx, "rmw_stage_r", args.rmw_stage_r)
     if args.wave_mb >= 0:
         B.agzo_set_option(ctx, "wave_bytes", args.wave_mb << 20)
+    if args.shard_tokens:     # rank p holds tokens [p m, (p + 1) m) of the batch
+        B.agzo_set_allreduce(ctx, B.torch_allreduce(), rank * cfg.m)
     work = algorithmic_work(cfg, r, args.alias_inputs)
     losses = torch.tensor([1.0, 0.999], dtype=torch.float64, device=dev)
     ghat = torch.zeros(1, device=dev)
@@ -383,6 +391,8 @@ def main():
                        "l2": "inputs larger than L2 (weights %.1f GB + activations %.1f GB per step)"
                              % (work["w_bytes"] / 1e9, work["x_bytes"] / 1e9),
                        "replicas": world, "device_status": B.status_string(status),
+                       "parallelism": ("token-sharded extraction (all-reduce of Y panels), replicated passes"
+                                       if args.shard_tokens else "independent replicas"),
                        "inputs": ("q/k/v and gate/up share one activation buffer per block" if args.alias_inputs
                                   else "one activation buffer per layer")},
             "phases_ms": {"extract": ms_extract, "perturb": ms_perturb, "restore_update": ms_update},
