@@ -31,10 +31,10 @@ import torch  # noqa: E402
 from paper_2601_17261_b200 import workloads as WL  # noqa: E402
 
 K_POWER = 3
-# DRAM bytes moved per algorithmic byte, from the ncu capture of each kernel on a 2-block
+# DRAM bytes moved per algorithmic byte, from the ncu capture of each kernel on a 4-block
 # slice of the 8B-shaped layer set (summaries under profiles/); traffic grows in proportion
 # to the activation bytes a launch sweeps.  Reset an entry to None when its kernel changes.
-TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (2.430687 + 0.040650) / 2.415919}
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (4.864893 + 0.012882) / 4.831838}
 EPS = 1e-3
 LR = 1e-6
 METRIC = "agzo_step_overhead_ms"
@@ -408,7 +408,7 @@ def main():
                          "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE["tc_xt_t_kernel"] * x_bytes_per_launch
                                      if tc_used and dom_n else None),
                          "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the "
-                                         "first 2 blocks of this workload, scaled by the X bytes a launch reads",
+                                         "first 4 blocks of this workload, scaled by the X bytes a launch reads",
                          "launches": dom_n, "avg_ms": dom_avg_ms,
                          "measured_with": "extract_streams=1, %.2f ms per step" % ms_step_one_stream},
             "gpu_launches": int(launches),
