@@ -94,14 +94,27 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
     if (lane == 0) {
       tmap_acquire(map_x);
       tmap_acquire(map_q);
-      for (int k = 0; k < nk; ++k) {
-        const int s = k % stages;
-        if (k >= stages && !mbar_wait(&sh.empty[s], ((k / stages) - 1) & 1)) { sh.failed = 1; break; }
-        uint8_t* a = tiles + (size_t)s * stage_bytes;
-        mbar_expect_tx(&sh.full[s], a_bytes + b_bytes);
-        tma_load_2d(a, map_x, k * kBoxK, t0, &sh.full[s]);
-        tma_load_2d(a + kTileBytes, map_x, k * kBoxK, t0 + 64, &sh.full[s]);
-        tma_load_2d(a + a_bytes, map_q, k * kBoxK, 0, &sh.full[s]);
+      // With four or more stages, two k-steps are issued together, box by box: the two 128-byte
+      // pieces of a token row then reach the memory system back to back (256 contiguous bytes per
+      // row instead of 128; 8B shapes, r = 16: T = X Q 20.6 -> 17.6 ms per step).  With three
+      // stages waiting for two free ones at a time costs more than it brings.
+      bool ok = true;
+      const int group = stages >= 4 ? 2 : 1;
+      for (int k = 0; k < nk && ok; k += group) {
+        const int n2 = min(group, nk - k);
+        uint8_t* a[2];
+        uint64_t* bar[2];
+        for (int u = 0; u < n2; ++u) {
+          const int kk = k + u, s = kk % stages;
+          if (kk >= stages && !mbar_wait(&sh.empty[s], ((kk / stages) - 1) & 1)) { sh.failed = 1; ok = false; break; }
+          a[u] = tiles + (size_t)s * stage_bytes;
+          bar[u] = &sh.full[s];
+          mbar_expect_tx(bar[u], a_bytes + b_bytes);
+        }
+        if (!ok) break;
+        for (int u = 0; u < n2; ++u) tma_load_2d(a[u], map_x, (k + u) * kBoxK, t0, bar[u]);
+        for (int u = 0; u < n2; ++u) tma_load_2d(a[u] + kTileBytes, map_x, (k + u) * kBoxK, t0 + 64, bar[u]);
+        for (int u = 0; u < n2; ++u) tma_load_2d(a[u] + a_bytes, map_q, (k + u) * kBoxK, 0, bar[u]);
       }
     }
   } else if (warp == 1) {

@@ -91,6 +91,7 @@ def test_calls_on_a_null_context_fail_cleanly(lib):
     assert lib.agzo_destroy(None) == B.AGZO_ERR_STATE
     assert lib.agzo_poll(None, None) == B.AGZO_ERR_STATE
     assert lib.agzo_set_option(None, b"extract_path", 1) == B.AGZO_ERR_STATE
+    assert lib.agzo_set_allreduce(None, B.ALLREDUCE_FN(), None, 0) == B.AGZO_ERR_STATE
 
 
 def test_missing_library_fails_loudly(monkeypatch):
