@@ -57,7 +57,8 @@ typedef enum agzo_status {
   AGZO_ERR_WORKSPACE = 4,     /* workspace missing, misaligned or too small for these layers */
   AGZO_ERR_STATE = 5,         /* call made on a destroyed / foreign context                 */
   AGZO_ERR_TIMEOUT = 6,       /* a bounded device-side wait ran out (reported by agzo_poll)  */
-  AGZO_ERR_CALLBACK = 7,      /* the loss callback of agzo_step returned non-zero           */
+  AGZO_ERR_CALLBACK = 7,      /* the loss callback of agzo_step, or the all-reduce callback
+                                 of a token-sharded extraction, returned non-zero            */
   AGZO_WARN_RANK_DEFICIENT = 100 /* some panel had a column with R_kk <= 1e-4 R_11; that
                                     column of V is zero (reported by agzo_poll)             */
 } agzo_status;
@@ -130,7 +131,9 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * "rmw_tc_panels" (column panels per work item, 1 or 2); "rmw_stage_r" 0 = when some layer's rank
  * exceeds 16 the split R operand of every 128-row tile is written once per pass to the scratch
  * area (d_out x 4 r' bytes per layer, r' = r rounded up to 16) and copied in by the pass instead of
- * being regenerated for every column panel, 1 = never, 2 = always;
+ * being regenerated for every column panel (later passes with the same seed and layers, i.e. the
+ * flip and the restore/update of the same step, find it there and skip the writing), 1 = never,
+ * 2 = always;
  * "share_inputs" 1 (default) = consecutive layers whose X is the same buffer (same pointer, pitch,
  * m, d_in: q/k/v or gate/up of a transformer block) are served by one sweep over X per product,
  * with identical results; 0 = every layer sweeps its X itself;

@@ -80,6 +80,9 @@ struct agzo_ctx {
   int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
   int extract_fused;       // 1: fused power-step kernel where a layer's shape allows it
   int share_inputs;        // 1: consecutive layers with the same X share the sweeps over it
+  // staged R images in scratch: valid for this seed until the plan changes or extraction uses the scratch
+  bool rimg_valid;
+  uint64_t rimg_seed;
   agzo_allreduce_fn allreduce;   // token-sharded extraction: sums a wave's Y panels over the ranks
   void* allreduce_user;
   int64_t token_offset;    // global index of this rank's first token
@@ -452,6 +455,7 @@ float* dev_coef(agzo_ctx* c) { return reinterpret_cast<float*>(c->ws + kCoefOffs
 // Makes the device tables describe `L`; uploads only when the descriptors changed.
 agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (same_layers(c, L, n)) return AGZO_OK;
+  c->rimg_valid = false;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
   PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels, c->rmw_stage_r,
@@ -517,10 +521,14 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   st = prepare(c, L, n, s);
   if (st != AGZO_OK) return st;
   if (c->plan.total_items > 0) {
-    Timed t(c, AGZO_KC_RMW_TC, s, c->plan.staged_r ? 2 : 1);
-    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->plan.max_r, c->plan.max_b_bytes, c->plan.max_row_tiles, c->plan.staged_r,
-                        c->rmw_tc_slots, c->rmw_tc_inflight, seed,
-                        coef, d_coef, dev_status(c), c->sm_count, s));
+    // the passes of one step share the seed, hence R: the images a pass staged serve the next ones
+    const bool fill = c->plan.staged_r && !(c->rimg_valid && c->rimg_seed == seed);
+    c->rimg_valid = false;
+    Timed t(c, AGZO_KC_RMW_TC, s, fill ? 2 : 1);
+    CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->plan.max_r,
+                        c->plan.max_b_bytes, c->plan.max_row_tiles, c->plan.staged_r, fill, c->rmw_tc_slots,
+                        c->rmw_tc_inflight, seed, coef, d_coef, dev_status(c), c->sm_count, s));
+    if (c->plan.staged_r) { c->rimg_valid = true; c->rimg_seed = seed; }
   }
   if (c->plan.total_tiles > 0) {
     Timed t(c, AGZO_KC_RMW, s);
@@ -545,7 +553,7 @@ const char* agzo_status_string(agzo_status s) {
     case AGZO_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case AGZO_ERR_STATE: return "invalid context";
     case AGZO_ERR_TIMEOUT: return "device-side wait ran out";
-    case AGZO_ERR_CALLBACK: return "loss callback failed";
+    case AGZO_ERR_CALLBACK: return "callback failed (loss or all-reduce)";
     case AGZO_WARN_RANK_DEFICIENT: return "rank-deficient activation panel";
   }
   return "unknown status";
@@ -597,6 +605,8 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->extract_streams = 2;
   c->extract_fused = 0;
   c->allreduce = nullptr;
+  c->rimg_valid = false;
+  c->rimg_seed = 0;
   c->allreduce_user = nullptr;
   c->token_offset = 0;
   c->share_inputs = 1;
@@ -756,6 +766,7 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
       if (!ctx->tc.available || !tc_eligible(h_layers[i])) return AGZO_ERR_UNSUPPORTED;
   st = prepare(ctx, h_layers, n, s);
   if (st != AGZO_OK) return st;
+  ctx->rimg_valid = false;   // extraction takes the scratch area
 
   const Plan& P = ctx->plan;
   // With two scratch regions, alternate waves run on two helper streams forked from the

@@ -266,11 +266,14 @@ constexpr int kCholThreads = 256;
 __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __restrict__ layers, int l0,
                                                             DevStatus* status) {
   const DevLayer& L = layers[l0 + blockIdx.x];
-  const int r = L.r;
-  __shared__ double S[AGZO_MAX_RANK][AGZO_MAX_RANK + 1];
+  const int r = L.r, rs = r + 1;        // rows of S and M are rs doubles apart (bank spread)
+  extern __shared__ __align__(16) double chol_smem[];
+  double* Sm = chol_smem;               // [r][rs]
+  double* Mm = chol_smem + r * rs;      // [r][rs]; copied to L.M at the end
   __shared__ int bad[AGZO_MAX_RANK];
   __shared__ double piv;
-  double* Mm = L.M;                     // [r][r], written and re-read by this block only
+#define S_(i, j) Sm[(i) * rs + (j)]
+#define M_(i, j) Mm[(i) * rs + (j)]
   const int tid = threadIdx.x;
   const int ti = tid >> 4, tj = tid & 15;          // 16 x 16 arrangement for the trailing update
   for (int p = tid; p < r * r; p += kCholThreads) {
@@ -279,31 +282,31 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
     if (j >= i)
       for (int c = 0; c < (L.gchunks + kGramGroup - 1) / kGramGroup; ++c)
         acc += L.Gpart[(long long)c * r * r + p];   // fixed order
-    S[i][j] = acc;
-    Mm[p] = 0.0;
+    S_(i, j) = acc;
+    M_(i, j) = 0.0;
   }
   __syncthreads();
   // right-looking Cholesky on the upper triangle; S is overwritten by R
   for (int k = 0; k < r; ++k) {
     if (tid == 0) {
-      const double d = S[k][k];
-      const double r11 = k == 0 ? 0.0 : S[0][0];
+      const double d = S_(k, k);
+      const double r11 = k == 0 ? 0.0 : S_(0, 0);
       int b = 0;
       if (!(d > 0.0)) b = 1;
       else if (k > 0 && sqrt(d) <= (double)kRankTol * r11) b = 1;
       bad[k] = b;
       piv = b ? 0.0 : sqrt(d);
-      S[k][k] = piv;
+      S_(k, k) = piv;
       if (b) atomicExch(&status->rank_deficient, 1);
     }
     __syncthreads();
     const double pk = piv;
-    for (int j = k + 1 + tid; j < r; j += kCholThreads) S[k][j] = pk > 0.0 ? S[k][j] / pk : 0.0;
+    for (int j = k + 1 + tid; j < r; j += kCholThreads) S_(k, j) = pk > 0.0 ? S_(k, j) / pk : 0.0;
     __syncthreads();
     for (int i = k + 1 + ti; i < r; i += 16) {
-      const double ski = S[k][i];
+      const double ski = S_(k, i);
       for (int j = k + 1 + tj; j < r; j += 16)
-        if (j >= i) S[i][j] -= ski * S[k][j];
+        if (j >= i) S_(i, j) -= ski * S_(k, j);
     }
     __syncthreads();
   }
@@ -313,13 +316,17 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
     if (!bad[k]) {
       for (int row = tid; row <= k; row += kCholThreads) {
         double acc = row == k ? 1.0 : 0.0;
-        for (int i = row; i < k; ++i) acc -= Mm[row * r + i] * S[i][k];
-        Mm[row * r + k] = acc / S[k][k];
+        for (int i = row; i < k; ++i) acc -= M_(row, i) * S_(i, k);
+        M_(row, k) = acc / S_(k, k);
       }
     }
     __syncthreads();
   }
+  for (int p = tid; p < r * r; p += kCholThreads) L.M[p] = M_(p / r, p % r);
+#undef S_
+#undef M_
 }
+size_t chol_smem_bytes(int r) { return (size_t)2 * r * (r + 1) * sizeof(double); }
 
 // ------------------------------------------------------------------ qr(Y), stage 3: Q = Y M
 // thread per column d, eight columns of Q at a time (M is upper triangular: column k needs Y's
@@ -393,7 +400,12 @@ cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStrea
       w.d_layers, w.l0, w.y_reduced);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  chol_kernel<<<nl, kCholThreads, 0, s>>>(w.d_layers, w.l0, d_status);
+  const size_t chol_bytes = chol_smem_bytes(w.max_r);
+  if (chol_bytes > 48 * 1024) {   // above the default limit of dynamic shared memory
+    e = cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chol_smem_bytes(AGZO_MAX_RANK));
+    if (e != cudaSuccess) return e;
+  }
+  chol_kernel<<<nl, kCholThreads, chol_bytes, s>>>(w.d_layers, w.l0, d_status);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   apply_kernel<<<dim3((w.max_din + 127) / 128, nl), 128, (size_t)w.max_r * ((w.max_r + 7) & ~7) * sizeof(double), s>>>(

@@ -503,11 +503,12 @@ size_t rmw_tc_image_bytes(const agzo_layer& a) {
 }
 
 cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
-                          int max_rp, int max_r, int max_b_bytes, int max_row_tiles, bool staged, int slots_wanted, int inflight,
+                          int max_rp, int max_r, int max_b_bytes, int max_row_tiles, bool staged, bool fill,
+                          int slots_wanted, int inflight,
                           uint64_t seed,
                           float coef, const float* d_coef, DevStatus* d_status, int sm_count, cudaStream_t s) {
   if (total_items <= 0) return cudaSuccess;
-  if (staged) {
+  if (staged && fill) {
     rmw_tc_fill_r_kernel<<<dim3((unsigned)max_row_tiles, (unsigned)n_layers), 256, 0, s>>>(d_layers, seed);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

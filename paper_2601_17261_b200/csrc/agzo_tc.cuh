@@ -37,9 +37,11 @@ cudaError_t rmw_tc_init();
 size_t rmw_tc_image_bytes(const agzo_layer& a);
 // shared-memory bytes of the B operand area that the layer's items need (after rmw_tc_shape)
 int rmw_tc_b_bytes(const DevLayer& D);
-// staged: the layers carry R images (DevLayer::rimg) that a fill kernel writes first
+// staged: the layers carry R images (DevLayer::rimg); fill: a fill kernel writes them first (not
+// needed when an earlier pass with the same seed and layers left them in place)
 cudaError_t launch_rmw_tc(const DevLayer* d_layers, const int* d_item_start, int n_layers, int total_items,
-                          int max_rp, int max_r, int max_b_bytes, int max_row_tiles, bool staged, int slots_wanted, int inflight,
+                          int max_rp, int max_r, int max_b_bytes, int max_row_tiles, bool staged, bool fill,
+                          int slots_wanted, int inflight,
                           uint64_t seed, float coef, const float* d_coef, DevStatus* d_status, int sm_count, cudaStream_t s);
 
 cudaError_t tc_fill_omega(const TcState& st, const ExtractWave& w, const DevLayer* h_dev,

@@ -120,6 +120,38 @@ def test_perturb_restore_update_match_oracle(d_out, d_in, r, storage, extra, lab
         assert bool((Vbuf[0] == 7).all() and (Vbuf[:, d_in:] == 7).all())
 
 
+def test_staged_R_is_rewritten_when_the_seed_changes_or_extraction_used_the_scratch():
+    d_out, d_in, r, layer_id = 300, 640, 24, 2
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=8, bf16=True)
+    X = WL.planted_activations(512, d_in, 16, seed=4, bf16=True)
+    Wd, _ = to_dev(W0, True)
+    Xd, _ = to_dev(X, True)
+    Vd = torch.zeros(r, d_in, device=DEV)
+    layers = [B.make_layer(W=Wd, X=Xd, V=Vd, r=r, layer_id=layer_id)]
+    with Ctx(layers) as ctx:
+        B.agzo_set_option(ctx, "rmw_path", 2)
+        B.agzo_extract_subspace(ctx, layers, 1, 2)
+        torch.cuda.synchronize()
+        Vh = Vd.cpu().numpy()
+
+        def one_pass(seed, c):
+            before = to_host(Wd)
+            B.agzo_perturb(ctx, layers, seed, c)
+            want = O.apply_direction(before, Vh, seed, layer_id, np.float32(c), "bf16")
+            assert_weights_match(to_host(Wd), want, "bf16",
+                                 floor=cancellation_floor(before, c, seed, layer_id, Vh, rel=2.0 ** -16))
+
+        one_pass(5, 1e-3)          # writes the images of seed 5
+        one_pass(5, -2e-3)         # finds them
+        one_pass(6, 1e-3)          # another seed: rewritten
+        one_pass(5, 1e-3)          # and back
+        B.agzo_extract_subspace(ctx, layers, 1, 2)     # the scratch now holds extraction's panels
+        torch.cuda.synchronize()
+        assert np.array_equal(Vd.cpu().numpy(), Vh)
+        one_pass(5, -1e-3)         # same seed as the last pass, yet rewritten
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+
+
 @pytest.mark.parametrize("stage", [1, 2])
 def test_tensor_core_pass_with_and_without_staged_R(stage):
     # stage 2: R tiles written to scratch by a fill kernel even at r = 8; stage 1: regenerated in the pass at r = 40
