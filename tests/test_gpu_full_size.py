@@ -121,3 +121,24 @@ def test_extraction_of_two_blocks_of_the_0p6b_shaped_set_with_shared_inputs():
         assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
         assert projector_distance(Vg, Vo) <= 1e-3
         assert np.abs(Vg - Vo).max() <= 1e-3
+
+
+def test_whole_batch_token_slabs_with_a_ragged_second_slab():
+    # 32 layers of d_in = 4096 have 1024 column blocks between them: the X^T T product then takes token
+    # slabs of up to 16384 tokens, here one full slab and a ragged one of 520.  The layers read one
+    # buffer but are not grouped (share_inputs off), so each sweeps it alone with its own Omega.
+    m, d_in, r, K, seed, n = 16384 + 520, 4096, 4, 1, 9, 32
+    X = WL.planted_activations(m, d_in, 16, seed=77, bf16=True)
+    Xd, _ = to_dev(X, True)
+    Vds = [torch.zeros(r, d_in, device=DEV) for _ in range(n)]
+    layers = [B.make_layer(X=Xd, V=Vds[i], r=r, layer_id=100 + i) for i in range(n)]
+    with Ctx(layers) as ctx:
+        B.agzo_set_option(ctx, "share_inputs", 0)
+        B.agzo_extract_subspace(ctx, layers, seed, K)
+        torch.cuda.synchronize()
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    for i in (0, 17, 31):
+        Vg = to_host(Vds[i])
+        Vo = O.extract_subspace(X, r, K, seed, 100 + i)
+        assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
+        assert projector_distance(Vg, Vo) <= 1e-3
