@@ -278,40 +278,48 @@ __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __r
 }
 
 // ---------------------------------------------------------------- Omega -> Tt (hi/lo), pads zero
-// local token t is row row0 + t of the whole batch's test matrix (see fill_omega_kernel)
-__global__ void tc_fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed, long long row0) {
+// Tt is [NB][m_pad] with the tokens contiguous, Omega's stream is row-major over (token, k): a
+// thread takes one token and eight consecutive k (at most three Philox blocks), so that for every
+// k a warp writes 32 neighbouring tokens.  Local token t is row row0 + t of the whole batch's
+// test matrix (see fill_omega_kernel).
+__global__ void __launch_bounds__(256) tc_fill_omega_kernel(const DevLayer* __restrict__ layers, int l0, uint64_t seed,
+                                                            long long row0) {
   const DevLayer& L = layers[l0 + blockIdx.y];
-  const long long n = (long long)L.m * L.r;
-  const long long e0 = row0 * L.r;
-  const long long b_end = (e0 + n + 3) >> 2;
+  const int r = L.r, NP = L.NP, groups = NP >> 3;
   const long long mp = L.m_pad;
-  const int r = L.r, NP = L.NP;
-  for (long long b = (e0 >> 2) + blockIdx.x * (long long)blockDim.x + threadIdx.x; b < b_end;
-       b += (long long)gridDim.x * blockDim.x) {
-    const float4 g = gaussian_block((uint64_t)b, L.layer_id, kTagOmega, seed);
-    const float gv[4] = {g.x, g.y, g.z, g.w};
+  const long long units = (long long)L.m * groups;
+  for (long long unit = blockIdx.x * 256ll + threadIdx.x; unit < units; unit += (long long)gridDim.x * 256) {
+    const int g = (int)(unit / L.m);
+    const long long t = unit - (long long)g * L.m;
+    const int nv = min(8, r - 8 * g);                 // live k of this group (the rest is padding)
+    float v[8];
 #pragma unroll
-    for (int lane = 0; lane < 4; ++lane) {
-      const long long e = 4 * b + lane - e0;
-      if (e >= 0 && e < n) {
-        const long long t = e / r;
-        const int k = (int)(e - t * r);
-        __nv_bfloat16 h, l;
-        split_bf16(gv[lane], &h, &l);
-        L.Tb[(long long)k * mp + t] = h;
-        L.Tb[(long long)(NP + k) * mp + t] = l;
+    for (int u = 0; u < 8; ++u) v[u] = 0.f;
+    if (nv > 0) {
+      const long long e_first = (row0 + t) * r + 8 * g;
+      const long long b0 = e_first >> 2;
+      const int off = (int)(e_first & 3);
+      const int nblk = (off + nv + 3) >> 2;
+      float x[12];
+      const float4 ga = gaussian_block((uint64_t)b0, L.layer_id, kTagOmega, seed);
+      float4 gb = make_float4(0.f, 0.f, 0.f, 0.f), gc = gb;
+      if (nblk > 1) gb = gaussian_block((uint64_t)(b0 + 1), L.layer_id, kTagOmega, seed);
+      if (nblk > 2) gc = gaussian_block((uint64_t)(b0 + 2), L.layer_id, kTagOmega, seed);
+      x[0] = ga.x; x[1] = ga.y; x[2] = ga.z; x[3] = ga.w;
+      x[4] = gb.x; x[5] = gb.y; x[6] = gb.z; x[7] = gb.w;
+      x[8] = gc.x; x[9] = gc.y; x[10] = gc.z; x[11] = gc.w;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float y = off == 0 ? x[u] : off == 1 ? x[u + 1] : off == 2 ? x[u + 2] : x[u + 3];
+        v[u] = u < nv ? y : 0.f;
       }
     }
-  }
-  const int pad = NP - r;
-  if (pad > 0) {
-    const long long np = (long long)pad * L.m;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < np;
-         i += (long long)gridDim.x * blockDim.x) {
-      const int k = r + (int)(i / L.m);
-      const long long t = i % L.m;
-      L.Tb[(long long)k * mp + t] = __float2bfloat16_rn(0.f);
-      L.Tb[(long long)(NP + k) * mp + t] = __float2bfloat16_rn(0.f);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      __nv_bfloat16 h, l;
+      split_bf16(v[u], &h, &l);
+      L.Tb[(long long)(8 * g + u) * mp + t] = h;
+      L.Tb[(long long)(NP + 8 * g + u) * mp + t] = l;
     }
   }
 }
@@ -428,8 +436,8 @@ bool tc_encode_maps(const TcState& st, const DevLayer& D, void* host_maps) {
 }
 
 cudaError_t tc_fill_omega(const TcState&, const ExtractWave& w, const DevLayer*, uint64_t seed, cudaStream_t s) {
-  const long long nb = (((long long)w.max_m * w.max_r + 3) >> 2) + 1;
-  int gx = (int)((nb + 255) / 256);
+  const long long units = (long long)w.max_m * ((w.max_r + 7) >> 3);
+  int gx = (int)((units + 255) / 256);
   if (gx > 1024) gx = 1024;
   if (gx < 1) gx = 1;
   tc_fill_omega_kernel<<<dim3(gx, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, seed, w.omega_row0);
