@@ -109,11 +109,13 @@ def test_two_token_shards_give_the_whole_batch_subspace(path, K):
 
 
 def test_many_layers_in_one_sharded_call_use_one_buffer_per_wave():
-    # equal split point for all layers of the call; several layers per wave, two waves
+    # equal split point for all layers of the call; several layers per wave, two waves; layers 1 and 2
+    # read the same buffer (as q and k of a block do) and are served by one sweep over it
     m, m0 = 1024, 512
-    specs = [(256, 4), (512, 8), (384, 8), (256, 2)]
+    specs = [(256, 4), (512, 8), (512, 6), (256, 2)]
     seed = 5
     Xs = [WL.planted_activations(m, d, 16, seed=60 + i, bf16=True) for i, (d, r) in enumerate(specs)]
+    Xs[2] = Xs[1]
     hub = HostAllReduce(2)
 
     def body(rank):
@@ -121,13 +123,16 @@ def test_many_layers_in_one_sharded_call_use_one_buffer_per_wave():
         stream = torch.cuda.Stream()
         keep, layers = [], []
         for i, ((d, r), X) in enumerate(zip(specs, Xs)):
-            Xd, _ = to_dev(np.ascontiguousarray(X[:m0] if rank == 0 else X[m0:]), True)
+            if i == 2:
+                Xd = keep[1][0]
+            else:
+                Xd, _ = to_dev(np.ascontiguousarray(X[:m0] if rank == 0 else X[m0:]), True)
             Vd = torch.zeros(r, d, device=DEV)
             keep.append((Xd, Vd))
             layers.append(B.make_layer(X=Xd, V=Vd, r=r, layer_id=i))
         torch.cuda.synchronize()
         with Ctx(layers) as ctx:
-            B.agzo_set_option(ctx, "wave_bytes", 2 * m0 * 512 * 2)      # two layers per wave at most
+            B.agzo_set_option(ctx, "wave_bytes", 800 * 1024)      # layers 0 to 2 (768 KiB of X), then layer 3
             B.agzo_set_allreduce(ctx, hub.fn(rank), rank * m0)
             B.agzo_extract_subspace(ctx, layers, seed, 2, stream=stream)
             stream.synchronize()
