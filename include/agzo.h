@@ -124,7 +124,7 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * tensor-core kernels (UNSUPPORTED at call time if a layer cannot use them), 3 = as 2 but
  * without the fused power-step kernel (T = X Q and Y = X^T T as two sweeps over X);
  * "rmw_path" selects the kernel of the in-place passes: 0 = automatic (bf16 weights with
- * 16-byte aligned rows and r >= "rmw_tc_min_rank", default 8, take the tensor-core kernel,
+ * 16-byte aligned rows and r >= "rmw_tc_min_rank", default 3, take the tensor-core kernel,
  * everything else the CUDA-core kernels), 1 = CUDA-core kernels only, 2 = tensor-core kernel
  * for every layer that allows it; tuning knobs of that kernel, 0 = chosen by rank:
  * "rmw_tc_slots" (shared-memory ring slots), "rmw_tc_inflight" (loads in flight per CTA),

@@ -569,7 +569,7 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 8, 0, 0, true, false, false, 2}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, false, false, 2}, &plan, &scratch);
   if (st != AGZO_OK) return st;
   st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, false, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
@@ -596,7 +596,7 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->last_cuda = 0;
   c->extract_path = 0;
   c->rmw_path = 0;
-  c->rmw_tc_min_rank = 8;
+  c->rmw_tc_min_rank = 3;   // measured: from r = 3 on the tensor-core pass is the faster one
   c->rmw_tc_slots = 0;
   c->rmw_tc_inflight = 0;
   c->rmw_tc_panels = 0;

@@ -210,7 +210,7 @@ def test_many_layers_one_launch_mixed_shapes_and_ranks():
             want = O.apply_direction(W0, Vh, 77, 100 + i, np.float32(2e-3), "bf16")
             assert_weights_match(to_host(devW[i][0]), want, "bf16",
                                  floor=cancellation_floor(W0, 2e-3, 77, 100 + i, Vh,
-                                                          rel=2.0 ** -16 if r >= 8 else 2.0 ** -20))
+                                                          rel=2.0 ** -16 if r >= 3 else 2.0 ** -20))
 
 
 def test_perturb_is_deterministic_and_regenerates_the_same_direction():
