@@ -3,7 +3,7 @@
 //
 // The CUDA-core kernel (agzo_rmw.cu) spends r + 1 fp32 FMAs per weight; from r = 16 on that is
 // more arithmetic than the FP32 pipes can do in the time HBM needs to stream the weight once in
-// and once out.  Here the product Delta = R A^T of a 128-row tile is one small tcgen05.mma chain
+// and once out, and measured it falls behind this kernel from r = 3 on.  Here the product Delta = R A^T of a 128-row tile is one small tcgen05.mma chain
 // (M = 128, N = the panel's columns, K = 4 * rp), its fp32 result waits in TMEM, and the only
 // per-weight work left for the CUDA cores is  w + c * delta  and the rounding to bf16.
 //
@@ -13,9 +13,11 @@
 // the parts, so the products are exact and summed in fp32; what is dropped is below 2^-17 of
 // each term.
 //
-// Work item = (layer, chunk of up to 8 row tiles, group of up to two adjacent column panels).
+// Work item = (layer, chunk of 8 or 32 row tiles, group of up to two adjacent column panels).
 // The R operand of a row tile serves every panel of the group, so R is regenerated once per
-// 128 x (2 * panel width) weights and the CTA streams up to 1 KiB of every weight row.
+// 128 x (2 * panel width) weights and the CTA streams up to 1 KiB of every weight row.  For
+// ranks above 16 the R operands are not regenerated at all: a fill kernel writes every tile's
+// operand image to scratch once per seed and the CTA copies it in (staged R).
 //
 // Data flow of one CTA (persistent, one per SM):
 //   loader thread      TMA-loads 128 x 64 boxes of W into a ring of shared-memory slots
