@@ -142,3 +142,42 @@ def test_whole_batch_token_slabs_with_a_ragged_second_slab():
         Vo = O.extract_subspace(X, r, K, seed, 100 + i)
         assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
         assert projector_distance(Vg, Vo) <= 1e-3
+
+
+def test_whole_8b_shaped_set_as_the_benchmark_runs_it_sampled_layers():
+    """The benchmark's own workload and launch configuration: all 252 layers of the Qwen3-8B-shaped
+    set resident (13.9 GB of weights, 43.5 GB of activations, generated on the device as bench.py
+    does), r = 16, K = 3, default options, one extraction and one pass over the whole set.  The
+    oracle recomputes sampled layers from the same bytes: the first and the last layer, a
+    down-projection (d_in = 12288) and layers from the middle (other waves, other streams)."""
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    torch.cuda.empty_cache()          # blocks cached by earlier tests count as used
+    free, _ = torch.cuda.mem_get_info()
+    if free < 75 * 2 ** 30:
+        pytest.skip("needs 75 GB of free device memory")
+    cfg = WL.QWEN3_8B
+    r, K, seed, eps = 16, 3, 123, 1e-3
+    dev = torch.device(DEV)
+    Ws, Xs, Vs, layers = bench.build_layer_set(cfg, r, dev)
+    sample = [0, 6, 101, 125, 251]
+    W_before = {i: to_host(Ws[i]) for i in sample}
+    arr = B.layer_array(layers)
+    with Ctx(layers) as ctx:
+        B.agzo_extract_subspace(ctx, layers, seed, K, arr=arr)
+        B.agzo_perturb(ctx, layers, seed, eps, arr=arr)
+        torch.cuda.synchronize()
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    for i in sample:
+        X = Xs[i].float().cpu().numpy()
+        Vg = to_host(Vs[i])
+        Vo = O.extract_subspace(X, r, K, seed, i)
+        assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5, i
+        assert projector_distance(Vg, Vo) <= 1e-3, i
+        want = O.apply_direction(W_before[i], Vg, seed, i, np.float32(eps), "bf16")
+        assert_weights_match(to_host(Ws[i]), want, "bf16",
+                             floor=cancellation_floor(W_before[i], eps, seed, i, Vg, 2.0 ** -16))
+    del Ws, Xs, Vs
+    torch.cuda.empty_cache()
