@@ -260,8 +260,13 @@ __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __rest
 
 // ------------------------------------------------------------------ qr(Y), stage 2: one block per layer
 // S = sum of partial Gram matrices; Cholesky S = R^T R (upper R, positive diagonal); a pivot
-// with R_kk <= kRankTol * R_11 marks a deficient column, which becomes zero.  M (upper
-// triangular) is built so that Q = Y M: column k of M solves R-columns by forward substitution.
+// with R_kk <= kRankTol * R_11 marks a deficient column, which becomes zero.  M = R^-1 (upper
+// triangular, deficient rows and columns zero) is built so that Q = Y M.
+//
+// One barrier per Cholesky step: step k updates the trailing matrix from the still unscaled row
+// k (a_ki a_kj / a_kk), and row k is divided by its pivot during step k + 1, which no longer
+// reads it.  The columns of M do not depend on one another, so four lanes share a column and all
+// columns are solved side by side (back substitution, the lanes splitting each dot product).
 constexpr int kCholThreads = 256;
 __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __restrict__ layers, int l0,
                                                             DevStatus* status) {
@@ -271,57 +276,70 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
   double* Sm = chol_smem;               // [r][rs]
   double* Mm = chol_smem + r * rs;      // [r][rs]; copied to L.M at the end
   __shared__ int bad[AGZO_MAX_RANK];
-  __shared__ double piv;
 #define S_(i, j) Sm[(i) * rs + (j)]
 #define M_(i, j) Mm[(i) * rs + (j)]
   const int tid = threadIdx.x;
   const int ti = tid >> 4, tj = tid & 15;          // 16 x 16 arrangement for the trailing update
+  const int ngroups = (L.gchunks + kGramGroup - 1) / kGramGroup;
   for (int p = tid; p < r * r; p += kCholThreads) {
     const int i = p / r, j = p - i * r;
     double acc = 0.0;
     if (j >= i)
-      for (int c = 0; c < (L.gchunks + kGramGroup - 1) / kGramGroup; ++c)
-        acc += L.Gpart[(long long)c * r * r + p];   // fixed order
+      for (int c = 0; c < ngroups; ++c) acc += L.Gpart[(long long)c * r * r + p];   // fixed order
     S_(i, j) = acc;
     M_(i, j) = 0.0;
   }
   __syncthreads();
-  // right-looking Cholesky on the upper triangle; S is overwritten by R
+  // right-looking Cholesky on the upper triangle; S is overwritten by R.  Every thread takes the
+  // pivot decision itself from the same numbers.
+  double r11 = 0.0, prev_piv = 0.0;
   for (int k = 0; k < r; ++k) {
+    const double d = S_(k, k);
+    bool b = !(d > 0.0);
+    const double sq = b ? 0.0 : sqrt(d);
+    if (!b && k > 0 && sq <= (double)kRankTol * r11) b = true;
+    const double pk = b ? 0.0 : sq;
+    if (k == 0) r11 = pk;
+    if (k > 0) {    // row k - 1 is final now: divide it by its pivot (nobody reads it in this step)
+      for (int j = k - 1 + tid; j < r; j += kCholThreads)
+        S_(k - 1, j) = j == k - 1 ? prev_piv : (prev_piv > 0.0 ? S_(k - 1, j) / prev_piv : 0.0);
+    }
     if (tid == 0) {
-      const double d = S_(k, k);
-      const double r11 = k == 0 ? 0.0 : S_(0, 0);
-      int b = 0;
-      if (!(d > 0.0)) b = 1;
-      else if (k > 0 && sqrt(d) <= (double)kRankTol * r11) b = 1;
-      bad[k] = b;
-      piv = b ? 0.0 : sqrt(d);
-      S_(k, k) = piv;
+      bad[k] = b ? 1 : 0;
       if (b) atomicExch(&status->rank_deficient, 1);
     }
-    __syncthreads();
-    const double pk = piv;
-    for (int j = k + 1 + tid; j < r; j += kCholThreads) S_(k, j) = pk > 0.0 ? S_(k, j) / pk : 0.0;
-    __syncthreads();
-    for (int i = k + 1 + ti; i < r; i += 16) {
-      const double ski = S_(k, i);
-      for (int j = k + 1 + tj; j < r; j += 16)
-        if (j >= i) S_(i, j) -= ski * S_(k, j);
-    }
-    __syncthreads();
-  }
-  // M column by column: M[row][k] = (delta_{row,k} - sum_{row<=i<k} M[row][i] R[i][k]) / R[k][k];
-  // a deficient column stays zero
-  for (int k = 0; k < r; ++k) {
-    if (!bad[k]) {
-      for (int row = tid; row <= k; row += kCholThreads) {
-        double acc = row == k ? 1.0 : 0.0;
-        for (int i = row; i < k; ++i) acc -= M_(row, i) * S_(i, k);
-        M_(row, k) = acc / S_(k, k);
+    if (!b) {
+      const double inv = 1.0 / d;
+      for (int i = k + 1 + ti; i < r; i += 16) {
+        const double t = S_(k, i) * inv;
+        for (int j = k + 1 + tj; j < r; j += 16)
+          if (j >= i) S_(i, j) -= t * S_(k, j);
       }
     }
+    prev_piv = pk;
     __syncthreads();
   }
+  for (int j = r - 1 + tid; j < r; j += kCholThreads) S_(r - 1, j) = prev_piv;   // the last row is its pivot alone
+  __syncthreads();
+  // M = R^-1 column by column, four lanes per column: m_k = 1 / R_kk, then for i = k-1 .. 0
+  // m_i = -(sum_{i<j<=k} R_ij m_j) / R_ii; a deficient index contributes nothing and gets zero
+  for (int c0 = 0; c0 < r; c0 += kCholThreads / 4) {
+    const int k = c0 + (tid >> 2), q = tid & 3;
+    const bool live = k < r && !bad[k < r ? k : 0];
+    if (live && q == 0) M_(k, k) = 1.0 / S_(k, k);
+    __syncwarp();
+    for (int i = r - 2; i >= 0; --i) {             // the same trip count for every lane of the warp
+      double part = 0.0;
+      const bool row = live && i < k && !bad[i];
+      if (row)
+        for (int j = i + 1 + q; j <= k; j += 4) part += S_(i, j) * M_(j, k);
+      part += __shfl_xor_sync(0xffffffffu, part, 1);
+      part += __shfl_xor_sync(0xffffffffu, part, 2);
+      if (row && q == 0) M_(i, k) = -part / S_(i, i);
+      __syncwarp();
+    }
+  }
+  __syncthreads();
   for (int p = tid; p < r * r; p += kCholThreads) L.M[p] = M_(p / r, p % r);
 #undef S_
 #undef M_
