@@ -220,6 +220,9 @@ def main():
                          "for a like-for-like step-overhead comparison")
     ap.add_argument("--blocks", type=int, default=0,
                     help="keep only the first N transformer blocks of the layer set (profiling-sized runs)")
+    ap.add_argument("--mode", type=int, default=0, choices=[0, 1],
+                    help="0: two-point step, three in-place passes (the benchmarked form).  1: Algorithm 2 as printed, "
+                         "one-sided difference, two passes (perturb, restore+update)")
     ap.add_argument("--shard-tokens", action="store_true",
                     help="every rank's activations are its own tokens of one batch of N x m tokens: extraction sums "
                          "the Y panels over the ranks (NCCL all-reduce through agzo_set_allreduce); the in-place "
@@ -290,9 +293,10 @@ def main():
         else:
             B.agzo_extract_subspace(ctx, layers, seed, K_POWER, arr=arr)
         B.agzo_perturb(ctx, layers, seed, EPS, arr=arr)
-        B.agzo_perturb(ctx, layers, seed, -2 * EPS, arr=arr)
-        B.agzo_ghat(ctx, losses[0:1], losses[1:2], EPS, 0, ghat)
-        B.agzo_restore_update(ctx, layers, seed, EPS, LR, 0, ghat, arr=arr)
+        if args.mode == 0:
+            B.agzo_perturb(ctx, layers, seed, -2 * EPS, arr=arr)
+        B.agzo_ghat(ctx, losses[0:1], losses[1:2], EPS, args.mode, ghat)
+        B.agzo_restore_update(ctx, layers, seed, EPS, LR, args.mode, ghat, arr=arr)
 
     def barrier():
         if dist is not None:
@@ -387,7 +391,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic",
             "data": "synthetic", "method": args.method,
             "config": {"workload": f"{cfg.name}: {len(layers)} layers, {cfg.n_params() / 1e9:.3f} G weights, "
-                                   f"m={cfg.m} tokens, r={r}, K={K_POWER}, eps={EPS}, two-point",
+                                   f"m={cfg.m} tokens, r={r}, K={K_POWER}, eps={EPS}, " + ("two-point" if args.mode == 0 else "one-sided"),
                        "l2": "inputs larger than L2 (weights %.1f GB + activations %.1f GB per step)"
                              % (work["w_bytes"] / 1e9, work["x_bytes"] / 1e9),
                        "replicas": world, "device_status": B.status_string(status),
