@@ -197,7 +197,7 @@ def whole_job_units(per_rank_units: float, world: int) -> float:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="agzo", choices=["agzo", "reference"])
     ap.add_argument("--workload", default=WL.QWEN3_8B.name, choices=sorted(WL.LAYER_SETS))
@@ -421,14 +421,13 @@ def main():
         if e2e:
             line["e2e"] = e2e
         if not args.no_cpu_baseline and world == 1:
-            Xh, Wh = host_block(cfg, 1)
-            # one layer of block 0 keeps the CPU leg within tens of seconds
+            Xh, Wh = host_block(cfg)
+            # one transformer block (every block has the same shapes): tens of seconds of CPU work
             t = oracle_block_seconds(cfg, r, Xh, Wh)
-            scale = sum(di * (cfg.m + do) for (_, di, do) in cfg.block) / (cfg.block[0][1] * (cfg.m + cfg.block[0][2]))
-            line["cpu_baseline"] = {"value": t * 1e3 * scale * cfg.n_blocks, "unit": "ms",
+            line["cpu_baseline"] = {"value": t * 1e3 * cfg.n_blocks, "unit": "ms",
                                     "cores": os.cpu_count(), "kind": "oracle",
-                                    "sample": f"layer 0.q of {len(layers)} layers timed ({t:.2f} s), scaled by "
-                                              f"elements touched to the whole set (x{scale * cfg.n_blocks:.1f})"}
+                                    "sample": f"block 0 ({len(cfg.block)} of {len(layers)} layers) timed ({t:.1f} s), "
+                                              f"time x{cfg.n_blocks} blocks"}
         print(json.dumps(line))
     B.agzo_destroy(ctx)
     if dist is not None:
