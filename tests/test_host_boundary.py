@@ -110,3 +110,46 @@ def test_make_layer_reads_strides_and_dtypes():
     assert (L.ldx, L.m, L.x_dtype, L.ldv, L.r, L.layer_id) == (16, 10, B.AGZO_F32, 16, 2, 5)
     with pytest.raises(TypeError):
         B.make_layer(W=W.to(torch.float16), V=V, r=2, layer_id=0)
+
+
+C_PROGRAM = r"""
+#include "agzo.h"
+#include <stdio.h>
+int main(void) {
+  agzo_layer L = {0};
+  size_t bytes = 0;
+  agzo_status s;
+  L.d_in = 256; L.d_out = 128; L.m = 512; L.r = 4; L.ldw = 256; L.ldx = 256; L.ldv = 256;
+  L.W = (void*)0x1000; L.X = (void*)0x2000; L.V = (float*)0x3000;
+  L.w_dtype = AGZO_BF16; L.x_dtype = AGZO_BF16;
+  s = agzo_workspace_bytes(&L, 1, &bytes);
+  printf("%d %lu %s\n", (int)s, (unsigned long)bytes, agzo_status_string(s));
+  L.r = AGZO_MAX_RANK + 1;
+  if (agzo_workspace_bytes(&L, 1, &bytes) != AGZO_ERR_INVALID_ARG) return 2;
+  if (agzo_set_allreduce(0, 0, 0, 0) != AGZO_ERR_STATE) return 3;
+  return s == AGZO_OK && bytes > 0 ? 0 : 1;
+}
+"""
+
+
+def test_header_is_plain_c_and_the_library_links_from_c(tmp_path, lib):
+    """The boundary is a C ABI: the header compiles as strict C99 without warnings and a C program
+    linked against the library can make the host-only calls (no GPU needed)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_agzo.c"
+    src.write_text(C_PROGRAM)
+    exe = tmp_path / "use_agzo"
+    libdir = os.path.dirname(B.LIB_PATH)
+    p = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(root, "include"),
+                        str(src), "-o", str(exe), "-L", libdir, "-lagzo", "-Wl,-rpath," + libdir],
+                       capture_output=True, text=True)
+    assert p.returncode == 0, p.stderr
+    run = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
+    assert run.returncode == 0, (run.stdout, run.stderr)
+    status, nbytes, text = run.stdout.split(maxsplit=2)
+    assert status == "0" and int(nbytes) > 0 and text.strip() == "ok"
