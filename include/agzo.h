@@ -310,6 +310,13 @@ agzo_status agzo_debug_philox(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, u
 agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, uint32_t tag,
                                 uint64_t first, uint64_t n, float* d_vals, void* stream);
 
+/* Exercises the bounded device-side wait that every pipeline of the tensor-core kernels uses:
+ * launches one small block that waits, with the library's own wait routine, on a barrier that
+ * nothing ever completes.  The wait gives up after its time limit (two seconds), the block
+ * records the condition in the status word and exits normally; the next agzo_poll returns
+ * AGZO_ERR_TIMEOUT and the context stays usable.  UNSUPPORTED without the tensor-core path. */
+agzo_status agzo_debug_wait_timeout(agzo_ctx* ctx, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

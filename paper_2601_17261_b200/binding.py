@@ -32,6 +32,7 @@ EXPORTS = [
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
     "agzo_extract_subspace_static", "agzo_fill_gaussian_basis", "agzo_set_allreduce",
+    "agzo_debug_wait_timeout",
 ]
 KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC, KC_FUSED_POWER = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
@@ -99,6 +100,7 @@ def lib() -> C.CDLL:
         "agzo_debug_gaussian": (i32, [vp, u64, u32, u32, u64, u64, vp, vp]),
         "agzo_read_counters": (i32, [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)]),
         "agzo_set_allreduce": (i32, [vp, ALLREDUCE_FN, vp, i64]),
+        "agzo_debug_wait_timeout": (i32, [vp, vp]),
         "agzo_extract_subspace_static": (i32, [vp, i64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                C.c_int32, u64, u32, vp, i64, vp, vp]),
     }
@@ -374,6 +376,10 @@ def agzo_perturb_dense(ctx: Context, w: torch.Tensor, seed: int, layer_id: int, 
                                     layer_id, scale,
                                     d_scale.data_ptr() if d_scale is not None else None,
                                     _stream_ptr(stream)), "agzo_perturb_dense")
+
+
+def agzo_debug_wait_timeout(ctx: Context, stream=None) -> None:
+    _check(lib().agzo_debug_wait_timeout(ctx.handle, _stream_ptr(stream)), "agzo_debug_wait_timeout")
 
 
 def agzo_debug_philox(ctx: Context, seed: int, layer_id: int, tag: int, first: int, n: int,

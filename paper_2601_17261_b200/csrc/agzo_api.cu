@@ -1023,4 +1023,12 @@ agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id,
   return AGZO_OK;
 }
 
+agzo_status agzo_debug_wait_timeout(agzo_ctx* ctx, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!ctx->tc.available) return AGZO_ERR_UNSUPPORTED;
+  CU(ctx, launch_debug_wait(dev_status(ctx), static_cast<cudaStream_t>(stream)));
+  return AGZO_OK;
+}
+
 }  // extern "C"

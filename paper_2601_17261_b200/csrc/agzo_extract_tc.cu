@@ -324,6 +324,20 @@ __global__ void __launch_bounds__(256) tc_fill_omega_kernel(const DevLayer* __re
   }
 }
 
+// ---------------------------------------------------------------- the bounded wait, on its own
+__global__ void debug_wait_kernel(DevStatus* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && !mbar_wait(&bar, 0)) {     // nobody arrives: the wait runs out
+    atomicExch(&status->timeout, 1);
+    atomicExch(&status->where, 100);
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -393,6 +407,11 @@ cudaError_t tc_init(TcState* st, int device) {
     if (e != cudaSuccess) { cudaGetLastError(); st->available = false; }
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_debug_wait(DevStatus* d_status, cudaStream_t s) {
+  debug_wait_kernel<<<1, 32, 0, s>>>(d_status);
+  return cudaGetLastError();
 }
 
 bool tc_eligible(const agzo_layer& a) {

@@ -33,6 +33,8 @@ bool rmw_tc_eligible(const agzo_layer& a);
 void rmw_tc_shape(const agzo_layer& a, int panels, bool staged, DevLayer* D);   // fills the rtc_* fields except item0 / wmap
 bool rmw_tc_encode_map(const TcState& st, const DevLayer& D, void* host_map);
 cudaError_t rmw_tc_init();
+// one block that waits on a barrier nothing completes, until the bounded wait gives up (test export)
+cudaError_t launch_debug_wait(DevStatus* d_status, cudaStream_t s);
 // bytes of the staged R operand images of one layer (every 128-row tile, K atoms of 16 KiB each)
 size_t rmw_tc_image_bytes(const agzo_layer& a);
 // shared-memory bytes of the B operand area that the layer's items need (after rmw_tc_shape)

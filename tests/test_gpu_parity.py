@@ -463,3 +463,28 @@ def test_empty_layer_list_and_argument_errors():
     assert B.lib().agzo_extract_subspace(small.handle, B.layer_array([big]), 1, 0, 3, None) == B.AGZO_ERR_WORKSPACE
     B.agzo_destroy(small)
     assert bool((W == 0).all())
+
+
+def test_a_device_side_wait_that_nothing_ends_gives_up_and_is_reported():
+    """Failure detection without a fault: the library's bounded wait, on a barrier that nobody
+    completes, returns after its time limit; the condition reaches the host through the status
+    word, and the context keeps working."""
+    import time
+    d_out, d_in, r, seed = 130, 256, 8, 3
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=1, bf16=True)
+    Vh = O.extract_subspace(WL.plain_activations(64, d_in, seed=2), r, 1, 3, 0)
+    Wd, _ = to_dev(W0, True)
+    Vd, _ = to_dev(Vh, False)
+    layers = [B.make_layer(W=Wd, V=Vd, r=r, layer_id=0)]
+    with Ctx(layers) as ctx:
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+        t0 = time.perf_counter()
+        B.agzo_debug_wait_timeout(ctx)
+        assert B.agzo_poll(ctx) == B.AGZO_ERR_TIMEOUT          # poll waits for the stream
+        assert 1.0 < time.perf_counter() - t0 < 20.0           # the limit is two seconds
+        assert B.agzo_poll(ctx) == B.AGZO_OK                   # reported once, then cleared
+        B.agzo_perturb(ctx, layers, seed, 1e-3)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    want = O.apply_direction(W0, Vh, seed, 0, np.float32(1e-3), "bf16")
+    assert_weights_match(to_host(Wd), want, "bf16",
+                         floor=cancellation_floor(W0, 1e-3, seed, 0, Vh, rel=2.0 ** -16))
