@@ -351,7 +351,9 @@ bool encode_2d(void* fn, void* out, const void* base, uint64_t inner, uint64_t o
   const cuuint32_t es[2] = {1, 1};
   CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
                                                    dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                                   // 256-byte promotion: the neighbouring 128 bytes of a row are
+                                                   // what the next box of the same rows reads
+                                                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   std::memcpy(out, &m, sizeof(m));
