@@ -34,7 +34,7 @@ K_POWER = 3
 # DRAM bytes moved per algorithmic byte, from the ncu capture of each kernel on a 4-block
 # slice of the 8B-shaped layer set (summaries under profiles/); traffic grows in proportion
 # to the activation bytes a launch sweeps.  Reset an entry to None when its kernel changes.
-TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (4.864893 + 0.012882) / 4.831838}
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (4.865842 + 0.012305) / 4.831838}
 EPS = 1e-3
 LR = 1e-6
 METRIC = "agzo_step_overhead_ms"
