@@ -155,8 +155,15 @@ def qr_positive(Y: np.ndarray):
 
     The paper writes [Q, ~] = qr(Y) without fixing signs; the low-rank direction R A^T
     depends on the basis and not only on its span, so the unique factorisation with a
-    positive diagonal is taken.  A column whose R_kk <= RANK_TOL * R_11 (a rank-deficient
-    panel) is returned as zero and reported.
+    positive diagonal is taken.
+
+    Rank deficiency (Algorithm 1 only assumes r << min(d_out, d_in, m) and says nothing
+    about it): column k is dependent on the columns before it when what is left of it after
+    they are projected out, R_kk, is at most RANK_TOL times the column's own length
+    ||y_k||.  Such a column is returned as zero and reported.  The test is relative to the
+    column itself, not to R_11: the columns of Y = H (H^T Q) carry the squared singular
+    values of H, and Section 3.2 reports rapidly decaying activation spectra, so a small
+    column is the normal case and says nothing about dependence.
     Returns (Q, R, deficient) with Q d x r float64.
     """
     Y = np.asarray(Y, dtype=np.float64)
@@ -166,6 +173,7 @@ def qr_positive(Y: np.ndarray):
     deficient = False
     for j in range(r):
         v = Y[:, j].copy()
+        own = np.sqrt(v @ v)
         for _ in range(2):
             for i in range(j):
                 c = Q[:, i] @ v
@@ -173,7 +181,7 @@ def qr_positive(Y: np.ndarray):
                 v -= c * Q[:, i]
         nrm = np.sqrt(v @ v)
         R[j, j] = nrm
-        if j > 0 and nrm <= RANK_TOL * R[0, 0] or nrm == 0.0:
+        if nrm <= RANK_TOL * own or nrm == 0.0:
             deficient = True
             continue
         Q[:, j] = v / nrm

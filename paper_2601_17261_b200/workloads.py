@@ -84,6 +84,36 @@ def planted_activations(m: int, d_in: int, p: int, seed: int, bf16: bool) -> np.
     return to_bf16_values(x) if bf16 else x
 
 
+def graded_activations(m: int, d_in: int, n_dirs: int, seed: int, bf16: bool, ratio: float = 2.0 ** -0.5,
+                       floor: float = 0.0) -> np.ndarray:
+    """Activations with a geometric spectrum: singular values sigma_k = sigma_0 * ratio^k over the first
+    n_dirs directions (random orthonormal singular vectors on both sides), entries of order one, plus
+    an optional isotropic noise floor of standard deviation `floor` per entry.  Stands in for the
+    rapidly decaying activation spectra of Section 3.2."""
+    rng = np.random.default_rng([seed, 0x5C])
+    U, _ = np.linalg.qr(rng.standard_normal((m, n_dirs)))
+    W, _ = np.linalg.qr(rng.standard_normal((d_in, n_dirs)))
+    s = ratio ** np.arange(n_dirs)
+    s = s * np.sqrt(m * d_in / np.sum(s * s))          # rms entry = 1
+    x = (U * s) @ W.T
+    if floor > 0.0:
+        x = x + floor * rng.standard_normal((m, d_in))
+    x = x.astype(np.float32)
+    return to_bf16_values(x) if bf16 else x
+
+
+def massive_activations(m: int, d_in: int, seed: int, bf16: bool, factor: float = 100.0,
+                        channel: int = 7, token: int = 11) -> np.ndarray:
+    """N(0,1) activations in which one channel (column) and one token (row) are `factor` times
+    larger than the rest: the outlier features and sink tokens of language models."""
+    rng = np.random.default_rng([seed, 0x5D])
+    x = rng.standard_normal((m, d_in))
+    x[:, channel % d_in] *= factor
+    x[token % m, :] *= factor
+    x = x.astype(np.float32)
+    return to_bf16_values(x) if bf16 else x
+
+
 def plain_activations(m: int, d_in: int, seed: int, bf16: bool = False) -> np.ndarray:
     rng = np.random.default_rng([seed, 0x59])
     x = rng.standard_normal((m, d_in)).astype(np.float32)

@@ -191,6 +191,58 @@ def test_rank_deficient_panel_yields_zero_columns():
     assert abs(info["V64"][0] @ info["V64"][1]) < 1e-10
 
 
+def test_rank_test_is_relative_to_the_column_itself():
+    # qr(Y) must not depend on the scale of a column: an independent column is kept however
+    # small it is next to the first one, a dependent column is dropped however large it is.
+    # (A test against R_11 fails both halves.)
+    rng = np.random.default_rng(7)
+    Y = rng.standard_normal((40, 4))
+    Qn, _ = _posqr(Y)
+    for scale in (1e-9, 1e-3, 1.0, 1e6):
+        Q, R, bad = O.qr_positive(Y * np.array([1.0, scale, 1.0, scale]))
+        assert not bad and np.abs(Q - Qn).max() < 1e-9
+    Yd = Y.copy()
+    Yd[:, 2] = 3.0 * Y[:, 0] - 2.0 * Y[:, 1]            # exactly dependent
+    for scale in (1e-6, 1.0, 1e13):
+        Q, R, bad = O.qr_positive(Yd * np.array([1.0, 1.0, scale, 1.0]))
+        assert bad and np.all(Q[:, 2] == 0.0)
+        assert np.abs(np.linalg.norm(Q[:, [0, 1, 3]], axis=0) - 1.0).max() < 1e-12
+
+
+def test_a_dominant_direction_does_not_cost_the_others():
+    # sigma_1 / sigma_2 = 1000 (an outlier feature): the columns of Y = H (H^T Q) then differ by
+    # 1e6 in length, yet Algorithm 1 returns r orthonormal columns spanning the top-r singular
+    # subspace.  (With the pivot compared to R_11 the second column would be zeroed.)
+    rng = np.random.default_rng(9)
+    m, d_in, r = 120, 48, 4
+    U, _ = np.linalg.qr(rng.standard_normal((m, d_in)))
+    Wt, _ = np.linalg.qr(rng.standard_normal((d_in, d_in)))
+    s = np.concatenate([[1000.0, 1.0, 0.5, 0.25], 0.01 * np.ones(d_in - 4)])
+    X = (U * s) @ Wt.T
+    V, info = O.extract_subspace(X, r, 3, seed=6, layer_id=1, return_info=True)
+    assert not info["deficient"]
+    V64 = info["V64"]
+    assert np.abs(V64 @ V64.T - np.eye(r)).max() < 1e-10
+    top = Wt[:, :r].T                                  # exact top-r right singular vectors
+    assert np.linalg.norm(V64.T @ V64 - top.T @ top) < 1e-6
+
+
+def test_graded_and_outlier_activations_keep_all_columns():
+    # decaying spectrum (sigma_k = 2^(-k/2)) and "massive activation" inputs: no column is
+    # dropped, the basis is orthonormal and captures nearly the energy of the exact top-r
+    Xg = WL.graded_activations(600, 160, 64, seed=3, bf16=True)
+    Xm = WL.massive_activations(600, 160, seed=4, bf16=True)
+    for X in (Xg, Xm):
+        _, _, vt = np.linalg.svd(X.astype(np.float64), full_matrices=False)
+        for r in (4, 16):
+            V, info = O.extract_subspace(X, r, 3, seed=2, layer_id=5, return_info=True)
+            assert not info["deficient"]
+            V64 = info["V64"]
+            assert np.abs(V64 @ V64.T - np.eye(r)).max() < 1e-10
+            best = np.linalg.norm(X.astype(np.float64) @ vt[:r].T) ** 2
+            assert np.linalg.norm(X.astype(np.float64) @ V64.T) ** 2 >= (1.0 - 1e-3) * best
+
+
 # ----------------------------------------------------------------------------- perturbation
 def test_direction_is_confined_to_the_subspace():
     d_out, d_in, r = 24, 40, 5
