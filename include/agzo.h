@@ -59,8 +59,9 @@ typedef enum agzo_status {
   AGZO_ERR_TIMEOUT = 6,       /* a bounded device-side wait ran out (reported by agzo_poll)  */
   AGZO_ERR_CALLBACK = 7,      /* the loss callback of agzo_step, or the all-reduce callback
                                  of a token-sharded extraction, returned non-zero            */
-  AGZO_WARN_RANK_DEFICIENT = 100 /* some panel had a column with R_kk <= 1e-4 R_11; that
-                                    column of V is zero (reported by agzo_poll)             */
+  AGZO_WARN_RANK_DEFICIENT = 100 /* some panel had a column that depends on the columns before
+                                    it (R_kk <= 1e-4 of the column's own length); that column
+                                    of V is zero (reported by agzo_poll)                    */
 } agzo_status;
 
 typedef enum agzo_dtype { AGZO_BF16 = 0, AGZO_F32 = 1 } agzo_dtype;
@@ -144,7 +145,10 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * streams forked from and joined to the caller's stream, so that one wave's short kernels
  * overlap the other's sweeps over X; 1 = waves strictly one after another;
  * "time_kernel_class" = one agzo_kernel_class whose launches get a CUDA event pair on the
- * caller's stream (0 = none), read back by agzo_read_counters.                           */
+ * caller's stream (0 = none), read back by agzo_read_counters;
+ * "debug_fail_step_call" = n (test aid, 0 = off): the n-th internal call of agzo_step
+ * (extract, perturb, [flip,] ghat, restore_update) returns AGZO_ERR_CUDA on the host before
+ * launching anything, so that the step's error path can be exercised without a fault.    */
 agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value);
 
 /* Token-sharded extraction over data-parallel ranks.  Algorithm 1 touches the activations only
@@ -250,8 +254,11 @@ agzo_status agzo_restore_update(agzo_ctx* ctx, const agzo_layer* h_layers, int n
 /* One AGZO iteration (Algorithm 2): loss(phase 0) -> extract -> perturb(+eps) ->
  * loss(phase 1) -> [mode 0: perturb(-2 eps) -> loss(phase 2)] -> ghat -> restore_update.
  * d_losses2 (device, 2 doubles) receives f_plus and f_other (f_minus or f0), d_ghat (device,
- * 1 float) receives g.  If the callback fails, the outstanding perturbation is removed
- * before ERR_CALLBACK returns.                                                           */
+ * 1 float) receives g.  Error behaviour: the step tracks where the weights sit
+ * (W + c*Delta); if the callback fails (ERR_CALLBACK) or any of the library's own calls
+ * after the first pass returns an error, the inverse pass of the outstanding c is enqueued
+ * before the error is returned, so the weights are back at W (up to the rounding of one
+ * pass).  A failure before the first pass leaves W untouched.                            */
 agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n,
                       const agzo_params* h_params, agzo_loss_fn loss, void* user,
                       double* d_losses2, float* d_ghat, void* stream);
@@ -282,7 +289,9 @@ agzo_status agzo_fill_gaussian_basis(agzo_ctx* ctx, const agzo_layer* h_layers, 
  * another framework owns (or has frozen) the allocator, a callback in which an allocation
  * would synchronise the device, a job whose memory is fixed up front.  X and V are still
  * the caller's.  The call itself performs no cudaMalloc / cudaFree and calls no library
- * routine that allocates.
+ * routine that allocates.  (The very first call on a device makes the CUDA runtime load the
+ * library's kernels, for which the driver may set device memory aside; from the second call
+ * on a device the free device memory is the same before and after a call.)
  *   X [m][ldx] (x_dtype), V [r][ldv] fp32 out, d_rank_deficient: optional device int32 that
  *   receives 1 when a panel column was zeroed (see AGZO_WARN_RANK_DEFICIENT), else 0.
  * Limit: the scratch of the problem must fit the array,

@@ -77,7 +77,7 @@ struct DevStatus {
   int pad;
 };
 
-constexpr float kRankTol = 1e-4f;
+constexpr double kRankTol = 1e-4;
 
 // ---------------------------------------------------------------- Philox4x32-10
 // Counter-based generator of Salmon et al. (SC'11).  key = step seed, counter =
@@ -137,16 +137,16 @@ cudaError_t launch_rmw(const DevLayer* d_layers, const int* d_tile_start, int n_
                        uint64_t seed, float coef, const float* d_coef, bool pair_update,
                        int sm_count, cudaStream_t s);
 cudaError_t launch_dense(void* w, long long n, int dtype, uint64_t seed, uint32_t layer_id,
-                         float scale, const float* d_scale, cudaStream_t s);
+                         float scale, const float* d_scale, int sm_count, cudaStream_t s);
 cudaError_t launch_fill_basis(const DevLayer* d_layers, int n_layers, int max_elems, uint64_t seed, cudaStream_t s);
 cudaError_t launch_ghat(const double* fp, const double* fo, float eps, int mode, float* g,
                         cudaStream_t s);
 cudaError_t launch_coef(const float* g, float eps, float lr, int kind, float* d_coef,
                         cudaStream_t s);
 cudaError_t launch_debug_philox(uint64_t seed, uint32_t layer, uint32_t tag, uint64_t first,
-                                uint64_t n, uint32_t* out, cudaStream_t s);
+                                uint64_t n, uint32_t* out, int sm_count, cudaStream_t s);
 cudaError_t launch_debug_gauss(uint64_t seed, uint32_t layer, uint32_t tag, uint64_t first,
-                               uint64_t n, float* out, cudaStream_t s);
+                               uint64_t n, float* out, int sm_count, cudaStream_t s);
 
 // extraction, CUDA-core fp32 path; layers [l0, l1) form one wave
 struct ExtractWave {

@@ -260,7 +260,10 @@ __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __rest
 
 // ------------------------------------------------------------------ qr(Y), stage 2: one block per layer
 // S = sum of partial Gram matrices; Cholesky S = R^T R (upper R, positive diagonal); a pivot
-// with R_kk <= kRankTol * R_11 marks a deficient column, which becomes zero.  M = R^-1 (upper
+// with R_kk <= kRankTol * ||y_k|| (what is left of column k after the columns before it are
+// projected out, against the column's own length sqrt(S_kk)) marks a dependent column, which
+// becomes zero.  The test is scale-free per column: the columns of Y = H (H^T Q) carry squared
+// singular values, so a short column is normal and says nothing about dependence.  M = R^-1 (upper
 // triangular, deficient rows and columns zero) is built so that Q = Y M.
 //
 // One barrier per Cholesky step: step k updates the trailing matrix from the still unscaled row
@@ -276,6 +279,7 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
   double* Sm = chol_smem;               // [r][rs]
   double* Mm = chol_smem + r * rs;      // [r][rs]; copied to L.M at the end
   __shared__ int bad[AGZO_MAX_RANK];
+  __shared__ double own[AGZO_MAX_RANK];   // S_kk before elimination: the squared length of column k
 #define S_(i, j) Sm[(i) * rs + (j)]
 #define M_(i, j) Mm[(i) * rs + (j)]
   const int tid = threadIdx.x;
@@ -288,18 +292,18 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
       for (int c = 0; c < ngroups; ++c) acc += L.Gpart[(long long)c * r * r + p];   // fixed order
     S_(i, j) = acc;
     M_(i, j) = 0.0;
+    if (i == j) own[i] = acc;
   }
   __syncthreads();
   // right-looking Cholesky on the upper triangle; S is overwritten by R.  Every thread takes the
   // pivot decision itself from the same numbers.
-  double r11 = 0.0, prev_piv = 0.0;
+  double prev_piv = 0.0;
   for (int k = 0; k < r; ++k) {
     const double d = S_(k, k);
     bool b = !(d > 0.0);
     const double sq = b ? 0.0 : sqrt(d);
-    if (!b && k > 0 && sq <= (double)kRankTol * r11) b = true;
+    if (!b && d <= kRankTol * kRankTol * own[k]) b = true;
     const double pk = b ? 0.0 : sq;
-    if (k == 0) r11 = pk;
     if (k > 0) {    // row k - 1 is final now: divide it by its pivot (nobody reads it in this step)
       for (int j = k - 1 + tid; j < r; j += kCholThreads)
         S_(k - 1, j) = j == k - 1 ? prev_piv : (prev_piv > 0.0 ? S_(k - 1, j) / prev_piv : 0.0);

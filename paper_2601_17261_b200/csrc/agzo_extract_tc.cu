@@ -99,6 +99,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
       // row instead of 128; 8B shapes, r = 16: T = X Q 20.6 -> 17.6 ms per step).  With three
       // stages waiting for two free ones at a time costs more than it brings.
       bool ok = true;
+      int issued = 0;            // k-steps whose loads have been issued
       const int group = stages >= 4 ? 2 : 1;
       for (int k = 0; k < nk && ok; k += group) {
         const int n2 = min(group, nk - k);
@@ -115,6 +116,10 @@ __global__ void __launch_bounds__(kTcThreads) tc_x_q_kernel(const DevLayer* __re
         for (int u = 0; u < n2; ++u) tma_load_2d(a[u], map_x, (k + u) * kBoxK, t0, bar[u]);
         for (int u = 0; u < n2; ++u) tma_load_2d(a[u] + kTileBytes, map_x, (k + u) * kBoxK, t0 + 64, bar[u]);
         for (int u = 0; u < n2; ++u) tma_load_2d(a[u] + a_bytes, map_q, (k + u) * kBoxK, 0, bar[u]);
+        issued = k + n2;
+      }
+      if (!ok || sh.failed) {    // leaving early: the copies in flight must land before the CTA goes away
+        for (int k = issued > stages ? issued - stages : 0; k < issued; ++k) mbar_wait(&sh.full[k % stages], (k / stages) & 1);
       }
     }
   } else if (warp == 1) {
@@ -215,6 +220,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __r
     if (lane == 0) {
       tmap_acquire(map_x);
       tmap_acquire(map_t);
+      int issued = 0;
       for (int k = 0; k < nk; ++k) {
         const int s = k % stages;
         if (k >= stages && !mbar_wait(&sh.empty[s], ((k / stages) - 1) & 1)) { sh.failed = 1; break; }
@@ -224,6 +230,10 @@ __global__ void __launch_bounds__(kTcThreads) tc_xt_t_kernel(const DevLayer* __r
         tma_load_2d(a, map_x, d0, tk, &sh.full[s]);
         tma_load_2d(a + kTileBytes, map_x, d0 + 64, tk, &sh.full[s]);
         tma_load_2d(a + a_bytes, map_t, tk, 0, &sh.full[s]);
+        issued = k + 1;
+      }
+      if (sh.failed) {           // leaving early: the copies in flight must land before the CTA goes away
+        for (int k = issued > stages ? issued - stages : 0; k < issued; ++k) mbar_wait(&sh.full[k % stages], (k / stages) & 1);
       }
     }
   } else if (warp == 1) {

@@ -420,10 +420,11 @@ __global__ void dense_kernel(T* w, long long n, uint64_t seed, uint32_t layer_id
 }
 
 cudaError_t launch_dense(void* w, long long n, int dtype, uint64_t seed, uint32_t layer_id,
-                         float scale, const float* d_scale, cudaStream_t s) {
+                         float scale, const float* d_scale, int sm_count, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
   const long long nb = (n + 3) >> 2;
-  const int grid = (int)((nb + 255) / 256 < 148 * 8 ? (nb + 255) / 256 : 148 * 8);
+  const long long cap = (long long)sm_count * 8;      // eight resident blocks of 256 threads per SM
+  const int grid = (int)((nb + 255) / 256 < cap ? (nb + 255) / 256 : cap);
   if (dtype == AGZO_BF16)
     dense_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((__nv_bfloat16*)w, n, seed, layer_id, scale, d_scale);
   else
@@ -502,16 +503,18 @@ __global__ void debug_gauss_kernel(uint64_t seed, uint32_t layer, uint32_t tag, 
   }
 }
 cudaError_t launch_debug_philox(uint64_t seed, uint32_t layer, uint32_t tag, uint64_t first,
-                                uint64_t n, uint32_t* out, cudaStream_t s) {
+                                uint64_t n, uint32_t* out, int sm_count, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  const int grid = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+  const uint64_t cap = (uint64_t)sm_count * 8;
+  const int grid = (int)((n + 255) / 256 < cap ? (n + 255) / 256 : cap);
   debug_philox_kernel<<<grid, 256, 0, s>>>(seed, layer, tag, first, n, out);
   return cudaGetLastError();
 }
 cudaError_t launch_debug_gauss(uint64_t seed, uint32_t layer, uint32_t tag, uint64_t first,
-                               uint64_t n, float* out, cudaStream_t s) {
+                               uint64_t n, float* out, int sm_count, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  const int grid = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+  const uint64_t cap = (uint64_t)sm_count * 8;
+  const int grid = (int)((n + 255) / 256 < cap ? (n + 255) / 256 : cap);
   debug_gauss_kernel<<<grid, 256, 0, s>>>(seed, layer, tag, first, n, out);
   return cudaGetLastError();
 }

@@ -67,6 +67,53 @@ def test_in_place_passes_on_a_full_size_layer(d_out, d_in, r):
         assert B.agzo_poll(ctx) == B.AGZO_OK
 
 
+# ---- the Qwen3-1.7B-shaped configuration at its own shapes: d_in 2048 / 6144, d_out up to 6144,
+# m = 16 x 1024 tokens, planted rank 64, r in {4, 8, 16}
+@pytest.mark.parametrize("d_in,r", [(2048, 4), (2048, 16), (6144, 8), (6144, 16)])
+def test_extraction_of_a_1p7b_shaped_layer(d_in, r):
+    cfg = WL.QWEN3_1P7B
+    X = WL.planted_activations(cfg.m, d_in, cfg.planted_rank, seed=d_in + r, bf16=True)
+    Xd, _ = to_dev(X, True)
+    Vd = torch.zeros(r, d_in, device=DEV)
+    layers = [B.make_layer(X=Xd, V=Vd, r=r, layer_id=11)]
+    with Ctx(layers) as ctx:
+        B.agzo_extract_subspace(ctx, layers, 3, 3)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    Vg = to_host(Vd)
+    Vo = O.extract_subspace(X, r, 3, 3, 11)
+    assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5
+    assert projector_distance(Vg, Vo) <= 1e-3
+    assert np.abs(Vg - Vo).max() <= 1e-3
+
+
+@pytest.mark.parametrize("d_out,d_in,r", [(6144, 2048, 4), (6144, 2048, 8), (6144, 2048, 16),
+                                           (2048, 6144, 4), (2048, 6144, 8), (2048, 6144, 16), (1024, 2048, 8)])
+def test_in_place_passes_on_a_1p7b_shaped_layer(d_out, d_in, r):
+    seed, layer_id, eps = 6, 4, 1e-3
+    W0 = WL.gaussian_weights(d_out, d_in, 0.02, seed=d_out + r, bf16=True)
+    Vh = O.extract_subspace(WL.plain_activations(256, d_in, seed=r), r, 1, 3, layer_id)
+    Wd, _ = to_dev(W0, True)
+    Vd, _ = to_dev(Vh, False)
+    layers = [B.make_layer(W=Wd, V=Vd, r=r, layer_id=layer_id)]
+    ghat = torch.tensor([-0.27], device=DEV)
+    rel = 2.0 ** -16                 # tensor-core pass (r >= 3)
+    with Ctx(layers) as ctx:
+        B.agzo_perturb(ctx, layers, seed, eps)
+        want = O.apply_direction(W0, Vh, seed, layer_id, np.float32(eps), "bf16")
+        assert_weights_match(to_host(Wd), want, "bf16", floor=cancellation_floor(W0, eps, seed, layer_id, Vh, rel))
+        cur = to_host(Wd)
+        B.agzo_perturb(ctx, layers, seed, -2 * eps)
+        want = O.apply_direction(cur, Vh, seed, layer_id, np.float32(-2 * eps), "bf16")
+        assert_weights_match(to_host(Wd), want, "bf16", floor=cancellation_floor(cur, 2 * eps, seed, layer_id, Vh, rel))
+        cur = to_host(Wd)
+        B.agzo_restore_update(ctx, layers, seed, eps, 1e-3, 0, ghat)
+        c = O.update_coefficient(eps, 1e-3, np.float32(-0.27), 0)
+        want = O.apply_direction(cur, Vh, seed, layer_id, c, "bf16")
+        assert_weights_match(to_host(Wd), want, "bf16", frac=tc_mismatch_bound(want, c, seed, layer_id, Vh),
+                             floor=cancellation_floor(cur, c, seed, layer_id, Vh, rel))
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+
+
 def test_every_layer_of_the_0p6b_shaped_set_in_one_grouped_launch():
     """All 196 layers of the Qwen3-0.6B-shaped set (0.44 G bf16 weights) perturbed by one call, every
     weight compared with the oracle; the layer shapes repeat per block, so the directions are

@@ -82,6 +82,42 @@ def test_callback_failure_restores_the_weights():
     assert np.abs(to_host(Wd) - W0).max() <= 1e-7       # back at W within fp32 rounding
 
 
+@pytest.mark.parametrize("mode,fail_at", [(0, 3), (0, 4), (0, 5), (1, 3), (1, 4)])
+def test_a_failing_library_call_inside_a_step_restores_the_weights(mode, fail_at):
+    # The failure is made on the host: the option lets the n-th internal call of agzo_step
+    # (1 extract, 2 perturb, 3 flip [mode 0] / ghat [mode 1], then ghat, restore+update) return an
+    # error before it launches anything.  No GPU fault is involved.  Whatever fails after the
+    # first pass, the step must leave W where it started.
+    X, Yt, W0 = WL.least_squares_problem(seed=2, d_in=64, d_out=32, m=128)
+    Xd, _ = to_dev(X, False)
+    Wd, _ = to_dev(W0, False)
+    Vd = torch.zeros(2, 64, device=DEV)
+    layers = [B.make_layer(W=Wd, X=Xd, V=Vd, r=2, layer_id=0)]
+    losses = torch.zeros(2, device=DEV, dtype=torch.float64)
+    ghat = torch.zeros(1, device=DEV)
+    seen = []
+    with Ctx(layers) as ctx:
+        B.agzo_set_option(ctx, "debug_fail_step_call", fail_at)
+        with pytest.raises(B.AgzoError) as e:
+            B.agzo_step(ctx, layers, seed=3, eps=1e-2, lr=1e-3, K=2, mode=mode,
+                        loss_fn=lambda phase, slot, stream: seen.append(phase),
+                        d_losses2=losses, d_ghat=ghat)
+        assert e.value.status == B.AGZO_ERR_CUDA
+        torch.cuda.synchronize()
+        moved = np.abs(to_host(Wd) - W0).max()
+        assert moved <= 1e-7, moved                      # back at W within fp32 rounding
+        # the context keeps working, and a step without the injected failure does move W
+        B.agzo_set_option(ctx, "debug_fail_step_call", 0)
+
+        def loss_fn(phase, slot, stream):
+            losses[slot] = 1.0 + 0.25 * slot
+
+        B.agzo_step(ctx, layers, seed=3, eps=1e-2, lr=1e-3, K=2, mode=mode, loss_fn=loss_fn,
+                    d_losses2=losses, d_ghat=ghat)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+    assert np.abs(to_host(Wd) - W0).max() > 1e-6
+
+
 def test_mlp_master_compute_pair_ten_steps():
     """Ten AGZO steps on the 8-layer MLP, seeds 0..9, checked in lock step.
 
