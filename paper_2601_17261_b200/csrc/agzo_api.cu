@@ -83,6 +83,7 @@ struct agzo_ctx {
   // staged R images in scratch: valid for this seed until the plan changes or extraction uses the scratch
   bool rimg_valid;
   uint64_t rimg_seed;
+  cudaStream_t rimg_stream;   // stream the images were written on: another stream refills them
   agzo_allreduce_fn allreduce;   // token-sharded extraction: sums a wave's Y panels over the ranks
   void* allreduce_user;
   int64_t token_offset;    // global index of this rank's first token
@@ -97,8 +98,10 @@ struct agzo_ctx {
   size_t h_stage_bytes;
   cudaEvent_t stage_ev;
   bool stage_pending;
+  cudaStream_t stage_stream;  // stream of the last table upload: a call on another stream waits for stage_ev
   TcState tc;
   // measurement aid: event pairs around the launches of one kernel class
+  int debug_fail_step_call;   // test option: the n-th internal call of agzo_step fails on the host, 0 = off
   int time_class;
   std::vector<cudaEvent_t> events;   // pairs: start, stop
   size_t events_used;
@@ -327,10 +330,17 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
 
   // extraction waves: consecutive layers whose activations fit the wave budget and whose
   // scratch fits the workspace
+  // layers whose power steps run in the fused kernel keep 2048-token slabs (a slab is that kernel's
+  // work item); the long slabs are for the layers that the two-sweep kernels serve
+  auto runs_fused = [&](const agzo_layer& a) {
+    return opts.extract_fused && extract_path != 1 && extract_path != 3 && tc_available && tc_eligible(a) && fused_eligible(a);
+  };
   long long column_blocks = 0;
   for (int k = 0; k < n; ++k)
-    if (has_x(L[k]) && extract_path != 1 && tc_available && tc_eligible(L[k])) column_blocks += (L[k].d_in + 127) / 128;
-  const bool long_slabs = column_blocks >= kLongSlabColumnBlocks && !opts.extract_fused;
+    if (has_x(L[k]) && extract_path != 1 && tc_available && tc_eligible(L[k]) && !runs_fused(L[k]))
+      column_blocks += (L[k].d_in + 127) / 128;
+  const bool long_slabs_any = column_blocks >= kLongSlabColumnBlocks;
+  auto long_slabs_for = [&](const agzo_layer& a) { return long_slabs_any && !runs_fused(a); };
   int i = 0;
   while (i < n) {
     if (!has_x(L[i])) {
@@ -350,8 +360,9 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       if (tc != wave_tc) break;      // a wave runs on one kind of kernel
       // a unit is one layer, or a run of consecutive layers that read the same X (one sweep serves all)
       int glen = 1, rows = tc ? tc_operand_rows(L[j].r) : 0;
-      if (tc && opts.share_inputs && !opts.extract_fused) {
+      if (tc && opts.share_inputs && !runs_fused(L[j])) {
         while (j + glen < n && has_x(L[j + glen]) && same_input(L[j], L[j + glen]) && tc_eligible(L[j + glen]) &&
+               !runs_fused(L[j + glen]) &&
                rows + tc_operand_rows(L[j + glen].r) <= 256) {
           rows += tc_operand_rows(L[j + glen].r);
           ++glen;
@@ -359,7 +370,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       }
       auto unit_need = [&](int len, int nrows) {
         size_t b = 0;
-        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, long_slabs, false);
+        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, long_slabs_for(L[j + g]), false);
         if (tc) b += tc_panel_bytes(L[j], nrows);
         return b;
       };
@@ -381,7 +392,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
           DevLayer& D = plan->dev[j + g];
           const agzo_layer& a = L[j + g];
           int slabs, slab_rows;
-          slab_shape(a, tc, long_slabs, &slabs, &slab_rows);
+          slab_shape(a, tc, long_slabs_for(a), &slabs, &slab_rows);
           const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
           const size_t gch = (d + 127) / 128;
           D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
@@ -454,7 +465,11 @@ float* dev_coef(agzo_ctx* c) { return reinterpret_cast<float*>(c->ws + kCoefOffs
 
 // Makes the device tables describe `L`; uploads only when the descriptors changed.
 agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
-  if (same_layers(c, L, n)) return AGZO_OK;
+  if (same_layers(c, L, n)) {
+    // the tables were uploaded on another stream: this one must not read them before they have landed
+    if (c->stage_pending && s != c->stage_stream) CU(c, cudaStreamWaitEvent(s, c->stage_ev, 0));
+    return AGZO_OK;
+  }
   c->rimg_valid = false;
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
@@ -497,6 +512,7 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
     CU(c, cudaMemcpyAsync(c->ws + kHeaderBytes, c->h_stage, lb + tb, cudaMemcpyHostToDevice, s));
     CU(c, cudaEventRecord(c->stage_ev, s));
     c->stage_pending = true;
+    c->stage_stream = s;
   }
   c->plan = std::move(plan);
   c->cached.assign(L, L + n);
@@ -522,13 +538,13 @@ agzo_status rmw_pass(agzo_ctx* c, const agzo_layer* L, int n, uint64_t seed, flo
   if (st != AGZO_OK) return st;
   if (c->plan.total_items > 0) {
     // the passes of one step share the seed, hence R: the images a pass staged serve the next ones
-    const bool fill = c->plan.staged_r && !(c->rimg_valid && c->rimg_seed == seed);
+    const bool fill = c->plan.staged_r && !(c->rimg_valid && c->rimg_seed == seed && c->rimg_stream == s);
     c->rimg_valid = false;
     Timed t(c, AGZO_KC_RMW_TC, s, fill ? 2 : 1);
     CU(c, launch_rmw_tc(dev_layers(c), dev_items(c, n), n, c->plan.total_items, c->plan.max_rp, c->plan.max_r,
                         c->plan.max_b_bytes, c->plan.max_row_tiles, c->plan.staged_r, fill, c->rmw_tc_slots,
                         c->rmw_tc_inflight, seed, coef, d_coef, dev_status(c), c->sm_count, s));
-    if (c->plan.staged_r) { c->rimg_valid = true; c->rimg_seed = seed; }
+    if (c->plan.staged_r) { c->rimg_valid = true; c->rimg_seed = seed; c->rimg_stream = s; }
   }
   if (c->plan.total_tiles > 0) {
     Timed t(c, AGZO_KC_RMW, s);
@@ -607,6 +623,8 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->allreduce = nullptr;
   c->rimg_valid = false;
   c->rimg_seed = 0;
+  c->rimg_stream = nullptr;
+  c->stage_stream = nullptr;
   c->allreduce_user = nullptr;
   c->token_offset = 0;
   c->share_inputs = 1;
@@ -618,6 +636,7 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->stage_pending = false;
   c->stage_ev = nullptr;
   c->time_class = 0;
+  c->debug_fail_step_call = 0;
   c->events_used = 0;
   c->launches = 0;
   cudaError_t e = cudaSetDevice(device);
@@ -700,6 +719,10 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
   } else if (std::strcmp(name, "wave_bytes") == 0) {
     if (value < 0) return AGZO_ERR_INVALID_ARG;
     ctx->wave_bytes = value;
+  } else if (std::strcmp(name, "debug_fail_step_call") == 0) {
+    if (value < 0 || value > 16) return AGZO_ERR_INVALID_ARG;
+    ctx->debug_fail_step_call = (int)value;
+    return AGZO_OK;
   } else if (std::strcmp(name, "time_kernel_class") == 0) {
     if (value < 0 || value > 9) return AGZO_ERR_INVALID_ARG;
     ctx->time_class = (int)value;
@@ -950,30 +973,41 @@ agzo_status agzo_step(agzo_ctx* ctx, const agzo_layer* h_layers, int n, const ag
   double* d_fother = d_losses2 + 1;
   float* d_g = d_ghat;
 
+  // The library knows where the weights sit at every moment: W0 + outstanding * Delta.  Whatever
+  // fails after the first pass -- the callback or one of the library's own calls -- the inverse of
+  // the outstanding perturbation is applied before the error is returned.
+  float outstanding = 0.f;
+  int call = 0;     // internal calls of this step, counted for the host-side fault injection of the tests
+  auto injected = [&]() { return ++call == ctx->debug_fail_step_call; };
+  auto fail = [&](agzo_status why) {
+    if (outstanding != 0.f) agzo_restore(ctx, h_layers, n, p->seed, outstanding, stream);
+    return why;
+  };
+
   // step 1: unperturbed forward (fills X), then Algorithm 1 per layer
   if (loss(user, stream, 0, d_fother) != 0) return AGZO_ERR_CALLBACK;
-  st = agzo_extract_subspace(ctx, h_layers, n, p->seed, p->K, stream);
+  st = injected() ? AGZO_ERR_CUDA : agzo_extract_subspace(ctx, h_layers, n, p->seed, p->K, stream);
   if (st != AGZO_OK) return st;
   // step 2: W + eps*Delta
-  st = agzo_perturb(ctx, h_layers, n, p->seed, p->eps, stream);
+  st = injected() ? AGZO_ERR_CUDA : agzo_perturb(ctx, h_layers, n, p->seed, p->eps, stream);
   if (st != AGZO_OK) return st;
-  if (loss(user, stream, 1, d_fplus) != 0) {
-    agzo_restore(ctx, h_layers, n, p->seed, p->eps, stream);
-    return AGZO_ERR_CALLBACK;
-  }
+  outstanding = p->eps;
+  if (loss(user, stream, 1, d_fplus) != 0) return fail(AGZO_ERR_CALLBACK);
   if (p->mode == 0) {
     // a pair is always rebuilt from the untouched master, so its flip is -eps, not -2 eps
-    st = agzo_perturb(ctx, h_layers, n, p->seed, any_pair ? -p->eps : -2.0f * p->eps, stream);
-    if (st != AGZO_OK) return st;
-    if (loss(user, stream, 2, d_fother) != 0) {
-      agzo_restore(ctx, h_layers, n, p->seed, -p->eps, stream);
-      return AGZO_ERR_CALLBACK;
-    }
+    st = injected() ? AGZO_ERR_CUDA
+                    : agzo_perturb(ctx, h_layers, n, p->seed, any_pair ? -p->eps : -2.0f * p->eps, stream);
+    if (st != AGZO_OK) return fail(st);
+    outstanding = -p->eps;
+    if (loss(user, stream, 2, d_fother) != 0) return fail(AGZO_ERR_CALLBACK);
   }
-  st = agzo_ghat(ctx, d_fplus, d_fother, p->eps, p->mode, d_g, stream);
-  if (st != AGZO_OK) return st;
+  st = injected() ? AGZO_ERR_CUDA : agzo_ghat(ctx, d_fplus, d_fother, p->eps, p->mode, d_g, stream);
+  if (st != AGZO_OK) return fail(st);
   // step 3: restore and update in one pass
-  return agzo_restore_update(ctx, h_layers, n, p->seed, p->eps, p->lr, p->mode, d_g, stream);
+  st = injected() ? AGZO_ERR_CUDA
+                  : agzo_restore_update(ctx, h_layers, n, p->seed, p->eps, p->lr, p->mode, d_g, stream);
+  if (st != AGZO_OK) return fail(st);
+  return AGZO_OK;
 }
 
 agzo_status agzo_fill_gaussian_basis(agzo_ctx* ctx, const agzo_layer* h_layers, int n, uint64_t seed,
@@ -1000,7 +1034,7 @@ agzo_status agzo_perturb_dense(agzo_ctx* ctx, void* w, int64_t n_elems, int dtyp
   if (n_elems < 0 || (n_elems > 0 && !w)) return AGZO_ERR_INVALID_ARG;
   if (dtype != AGZO_BF16 && dtype != AGZO_F32) return AGZO_ERR_UNSUPPORTED;
   ctx->launches += 1;
-  CU(ctx, launch_dense(w, n_elems, dtype, seed, layer_id, scale, d_scale,
+  CU(ctx, launch_dense(w, n_elems, dtype, seed, layer_id, scale, d_scale, ctx->sm_count,
                        static_cast<cudaStream_t>(stream)));
   return AGZO_OK;
 }
@@ -1010,7 +1044,7 @@ agzo_status agzo_debug_philox(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, u
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
   if (n > 0 && !d_words) return AGZO_ERR_INVALID_ARG;
-  CU(ctx, launch_debug_philox(seed, layer_id, tag, first, n, d_words, static_cast<cudaStream_t>(stream)));
+  CU(ctx, launch_debug_philox(seed, layer_id, tag, first, n, d_words, ctx->sm_count, static_cast<cudaStream_t>(stream)));
   return AGZO_OK;
 }
 
@@ -1019,7 +1053,7 @@ agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id,
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
   if (n > 0 && !d_vals) return AGZO_ERR_INVALID_ARG;
-  CU(ctx, launch_debug_gauss(seed, layer_id, tag, first, n, d_vals, static_cast<cudaStream_t>(stream)));
+  CU(ctx, launch_debug_gauss(seed, layer_id, tag, first, n, d_vals, ctx->sm_count, static_cast<cudaStream_t>(stream)));
   return AGZO_OK;
 }
 

@@ -35,6 +35,8 @@
 // word and the CTA leaves through the common exit (copies drained, cluster barrier, TMEM freed).
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "agzo_ptx.cuh"
 #include "agzo_tc.cuh"
 
@@ -51,15 +53,17 @@ constexpr int kMBlocks = kSliceCols / 128; // M blocks of phase C
 constexpr int kSlotBytes = 16 * 1024;      // [64 tokens][128 columns] as two boxes of 64 columns
 constexpr int kBoxBytes = 8 * 1024;
 constexpr int kMaxRing = 12;
-constexpr int kRsFloats = 72 * 16;         // C * ceil(64 / C) <= 72 rows of up to 16 floats
+constexpr int kRsFloats = 1792;            // C * ceil(8 / C) * 8 * NP floats at most (C = 7, NP = 16)
 constexpr uint32_t kFzTmemCols = 256;
+constexpr int kLook = 1;                   // phase A runs this many tiles ahead of phase C
+constexpr int kBuf = kLook + 1;            // T partial / exchange / T operand buffers in rotation
 
 struct FzShared {
   uint64_t x_full[kMaxRing], x_empty[kMaxRing];
   uint64_t qb_full, qb_empty;
-  uint64_t tp_full[2], tp_empty[2];     // T partial in TMEM
-  uint64_t tt_full[2], tt_empty[2];     // T operand in shared memory
-  uint64_t rs_full[2], ag_full[2];      // exchange: contributions to my rows have landed / the summed T has landed
+  uint64_t tp_full[kBuf], tp_empty[kBuf];     // T partial in TMEM
+  uint64_t tt_full[kBuf];                     // T operand in shared memory: the owners' sums have landed
+  uint64_t rs_full[kBuf];                     // exchange: the contributions to the rank indices I own have landed
   uint64_t y_full, y_free;
   uint32_t tmem_base;
   int failed;
@@ -93,7 +97,7 @@ __device__ __forceinline__ uint32_t swz(int i, int j) {
 }
 
 __global__ void __launch_bounds__(kFzThreads, 1)
-fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, int ring, DevStatus* status) {
+fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, int ring, int pf, DevStatus* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ FzShared sh;
@@ -106,17 +110,16 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
   uint8_t* sQ = sX + (size_t)ring * kSlotBytes;
   // NB is a per-layer quantity; the regions are sized for NB = 32
   uint8_t* sTt = sQ + 8 * 32 * 128;
-  float* sRs = reinterpret_cast<float*>(sTt + 2 * 32 * 128);    // 2 x [C][rows_per][NP] floats
-  float* sAg = sRs + 2 * kRsFloats;                               // 2 x [64][16] floats
-  const int rows_per = (kTT + C - 1) / C;                         // token rows of a tile that one CTA sums
+  float* sRs = reinterpret_cast<float*>(sTt + kBuf * 32 * 128);  // kBuf x [C][cpo][8][NP] floats
+  uint8_t* sStage = reinterpret_cast<uint8_t*>(sRs + kBuf * kRsFloats);   // 512 bytes per epilogue warp
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < ring; ++s) { mbar_init(&sh.x_full[s], 1); mbar_init(&sh.x_empty[s], 1); }
     mbar_init(&sh.qb_full, 1); mbar_init(&sh.qb_empty, 1);
-    for (int p = 0; p < 2; ++p) {
+    for (int p = 0; p < kBuf; ++p) {
       mbar_init(&sh.tp_full[p], 1); mbar_init(&sh.tp_empty[p], 4);
-      mbar_init(&sh.tt_full[p], 4); mbar_init(&sh.tt_empty[p], 1);
-      mbar_init(&sh.rs_full[p], 1); mbar_init(&sh.ag_full[p], 1);
+      mbar_init(&sh.tt_full[p], 1);
+      mbar_init(&sh.rs_full[p], 1);
     }
     mbar_init(&sh.y_full, 1); mbar_init(&sh.y_free, 4);
     sh.failed = 0;
@@ -154,11 +157,15 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
           const int t0 = it.t_begin + tile * kTT;
           for (int b = 0; b < mb; ++b, ++ns) {
             const int s = ns % ring, u = ns / ring;
-            if (u > 0 && !mbar_wait(&sh.x_empty[s], (u - 1) & 1)) { ok = false; break; }
+            if (u > 0 && !mbar_wait_spin(&sh.x_empty[s], (u - 1) & 1)) { ok = false; break; }
             uint8_t* slot = sX + (size_t)s * kSlotBytes;
             mbar_expect_tx(&sh.x_full[s], kSlotBytes);
             tma_load_2d(slot, map_x, col0 + 128 * b, t0, &sh.x_full[s]);
             tma_load_2d(slot + kBoxBytes, map_x, col0 + 128 * b + 64, t0, &sh.x_full[s]);
+            if (tile + pf < it.ntiles) {     // the tile `pf` steps ahead starts its way from DRAM to L2 now
+              tma_prefetch_2d(map_x, col0 + 128 * b, t0 + pf * kTT);
+              tma_prefetch_2d(map_x, col0 + 128 * b + 64, t0 + pf * kTT);
+            }
           }
         }
       }
@@ -168,13 +175,17 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {
       // ------------------------------------------------ MMA issuer
+      // All 32 lanes run this loop and one elected lane issues (mma_bf16_if): the descriptors then
+      // stay warp-uniform values, which is what keeps an instruction at its hardware cost.
+      const uint32_t go = elect_one();
       int na = 0, nc = 0;      // slots consumed by phase A / phase C
       int ta = 0, tcn = 0;     // tiles issued in phase A / phase C
       int ic = 0;
       bool ok = true;
       FzItem it;
+      const uint32_t sq_addr = smem_u32(sQ), sx_addr = smem_u32(sX), stt_addr = smem_u32(sTt);
       for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters, ++ic) {
         const DevLayer& L = *it.L;
         const int NB = L.NB;
@@ -184,58 +195,58 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         const uint32_t idesc_a = instr_desc(64, NB, 0, 0);
         const uint32_t idesc_c = instr_desc(128, NB, 1, 0);      // A = resident X boxes read as X^T
         const uint32_t tp_col = (uint32_t)(kMBlocks * NB);       // T partials sit after the Y accumulators
-        if (!mbar_wait(&sh.qb_full, ic & 1)) { ok = false; break; }
-        if (ic > 0 && !mbar_wait(&sh.y_free, (ic - 1) & 1)) { ok = false; break; }
-        for (int step = 0; step <= it.ntiles && ok; ++step) {
+        if (!mbar_wait_warp(&sh.qb_full, ic & 1)) { ok = false; break; }
+        if (ic > 0 && !mbar_wait_warp(&sh.y_free, (ic - 1) & 1)) { ok = false; break; }
+        for (int step = 0; step < it.ntiles + kLook && ok; ++step) {
           if (step < it.ntiles) {
             // phase A of tile `step`
-            const int p = ta & 1, u2 = ta >> 1;
-            if (u2 > 0 && !mbar_wait(&sh.tp_empty[p], (u2 - 1) & 1)) { ok = false; break; }
-            bool first = true;
+            const int p = ta % kBuf, u2 = ta / kBuf;
+            if (u2 > 0 && !mbar_wait_warp(&sh.tp_empty[p], (u2 - 1) & 1)) { ok = false; break; }
+            const uint32_t d_tp = tmem + tp_col + (uint32_t)(p * NB);
+            uint32_t acc = 0u;
             for (int b = 0; b < mb && ok; ++b, ++na) {
               const int s = na % ring, u = na / ring;
-              if (!mbar_wait(&sh.x_full[s], u & 1)) { ok = false; break; }
+              if (!mbar_wait_warp(&sh.x_full[s], u & 1)) { ok = false; break; }
               tc_fence_after();
-              const uint32_t slot = smem_u32(sX + (size_t)s * kSlotBytes);
+              const uint32_t slot = sx_addr + (uint32_t)s * kSlotBytes;
               for (int half = 0; half < 2; ++half) {
                 if (128 * b + 64 * half >= live) break;          // box beyond d_in: its Q box was never loaded
-                const uint32_t xa = slot + half * kBoxBytes;
-                const uint32_t qb = smem_u32(sQ) + (uint32_t)(2 * b + half) * q_box;
+                const uint64_t xd = smem_desc(slot + half * kBoxBytes, 0, 1024);
+                const uint64_t qd = smem_desc(sq_addr + (uint32_t)(2 * b + half) * q_box, 0, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                  mma_bf16(tmem + tp_col + (uint32_t)(p * NB), smem_desc(xa + kk * 32, 0, 1024),
-                           smem_desc(qb + kk * 32, 0, 1024), idesc_a, first ? 0u : 1u);
-                  first = false;
+                for (int kk = 0; kk < 4; ++kk) {                 // 16 columns = 32 bytes = 2 descriptor units further
+                  mma_bf16_if(go, d_tp, xd + (uint64_t)(2 * kk), qd + (uint64_t)(2 * kk), idesc_a, acc);
+                  acc = 1u;
                 }
               }
             }
             if (!ok) break;
-            mma_commit(&sh.tp_full[p]);
-            if (step == it.ntiles - 1) mma_commit(&sh.qb_empty);   // last use of this item's Q slice
+            mma_commit_if(go, &sh.tp_full[p]);
+            if (step == it.ntiles - 1) mma_commit_if(go, &sh.qb_empty);   // last use of this item's Q slice
             ++ta;
           }
-          if (step >= 1) {
-            // phase C of tile `step - 1`
-            const int p = tcn & 1, u2 = tcn >> 1;
-            if (!mbar_wait(&sh.tt_full[p], u2 & 1)) { ok = false; break; }
+          if (step >= kLook) {
+            // phase C of tile `step - kLook`
+            const int p = tcn % kBuf, u2 = tcn / kBuf;
+            if (!mbar_wait_cluster_warp(&sh.tt_full[p], u2 & 1)) { ok = false; break; }
+            fence_proxy_async();      // the operand was written by generic-proxy stores of the owners
             tc_fence_after();
-            const uint32_t tt = smem_u32(sTt + (size_t)p * 32 * 128);
+            const uint64_t td = smem_desc(stt_addr + (uint32_t)p * 32u * 128u, 0, 1024);
             for (int b = 0; b < mb; ++b, ++nc) {
               const int s = nc % ring;
-              const uint32_t slot = smem_u32(sX + (size_t)s * kSlotBytes);
+              // 16 tokens = two 8-row swizzle atoms = 2048 bytes = 128 descriptor units further down both boxes
+              const uint64_t xd = smem_desc(sx_addr + (uint32_t)s * kSlotBytes, kBoxBytes, 1024);
+              const uint32_t d_y = tmem + (uint32_t)(b * NB);
 #pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                // 16 tokens = two 8-row swizzle atoms = 2048 bytes further down both boxes
-                mma_bf16(tmem + (uint32_t)(b * NB), smem_desc(slot + kk * 2048, kBoxBytes, 1024),
-                         smem_desc(tt + kk * 32, 0, 1024), idesc_c, (step > 1 || kk > 0) ? 1u : 0u);
-              }
-              mma_commit(&sh.x_empty[s]);
+              for (int kk = 0; kk < 4; ++kk)
+                mma_bf16_if(go, d_y, xd + (uint64_t)(128 * kk), td + (uint64_t)(2 * kk), idesc_c,
+                            (step > kLook || kk > 0) ? 1u : 0u);
+              mma_commit_if(go, &sh.x_empty[s]);
             }
-            mma_commit(&sh.tt_empty[p]);
             ++tcn;
           }
         }
-        if (ok) mma_commit(&sh.y_full);
+        if (ok) mma_commit_if(go, &sh.y_full);
       }
       if (!ok) sh.failed = 1;
     }
@@ -256,47 +267,54 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       const int live = min(kSliceCols, L.d_in - col0);
       const int mb = (live + 127) / 128;
       const uint32_t tp_col = (uint32_t)(kMBlocks * NB);
-      const int hn = NP >> 1;               // values of a T row that one thread sums: NP/2
+      const int cpo = (kTT / 8 + C - 1) / C;   // token groups of a tile per owner, at most
       for (int tile = 0; tile < it.ntiles && ok; ++tile, ++te) {
-        const int p = te & 1, u2 = te >> 1;
-        if (p != grp) continue;
-        ok = mbar_wait(&sh.tp_full[p], u2 & 1);
+        const int p = te % kBuf, u2 = te / kBuf;
+        if ((te & 1) != grp) continue;
+        ok = mbar_wait_spin(&sh.tp_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        // an M = 64 accumulator keeps row 16q + i in lane 32q + i for i < 16; lanes 16..31 of a warp hold nothing
+        // an M = 64 accumulator keeps row 16q + i in lane 32q + i for i < 16; lanes 16..31 of a warp hold nothing.
+        // The buffer's NB columns are [hi parts | lo parts]: one load of up to 32 columns brings both.
         float tsum[16];
-#pragma unroll
-        for (int kq = 0; kq < 2; ++kq) {
-          if (kq * 8 < NP) {
-            float hi[8], lo[8];
-            tmem_ld8(tmem + lane_off + tp_col + (uint32_t)(p * NB + kq * 8), hi);
-            tmem_ld8(tmem + lane_off + tp_col + (uint32_t)(p * NB + NP + kq * 8), lo);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) tsum[kq * 8 + j] = hi[j] + lo[j];
-          } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) tsum[kq * 8 + j] = 0.f;
+        {
+          uint32_t z[32];
+          if (NB == 32) {
+            tmem_ld32_issue(tmem + lane_off + tp_col + (uint32_t)(p * NB), z);
+          } else {            // NB = 16: the upper 16 registers are not used
+            tmem_ld16_issue(tmem + lane_off + tp_col + (uint32_t)(p * NB), z);
           }
+          tmem_ld_wait();
+#pragma unroll
+          for (int k = 0; k < 16; ++k)
+            tsum[k] = NB == 32 ? __uint_as_float(z[k]) + __uint_as_float(z[16 + k])
+                               : (k < 8 ? __uint_as_float(z[k]) + __uint_as_float(z[8 + k]) : 0.f);
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.tp_empty[p]);
         // Exchange, two one-way hops through st.async (data and its completion travel together):
-        //   reduce-scatter  row R of my partial goes to the CTA that owns R (rows_per rows each);
-        //   all-gather      the owner adds the C contributions in rank order and sends the sum to everyone.
-        // No buffer needs a "free" signal: a peer can only send tile i+2's data after it has received
-        // my tile-i sums, which I send after consuming the tile-i contributions.
-        float* rs = sRs + p * kRsFloats;          // [C sources][rows_per][NP]
-        float* ag = sAg + p * (kTT * 16);         // [64][NP]
-        const int my_rows = max(0, min(rows_per, kTT - rank * rows_per));
+        //   reduce-scatter  the tile's tokens are owned in groups of eight, group j by the CTA of rank j mod C:
+        //                   every CTA sends the owner its partial sums of those rows of T;
+        //   all-gather      the owner adds the C contributions in rank order, splits the sums into bf16 hi and
+        //                   lo parts and writes them straight into the T operand of every CTA of the cluster:
+        //                   eight tokens of one operand row are one 16-byte piece.  The bytes are counted on
+        //                   the receiver's tt_full barrier, which is what its MMA warp waits for.
+        // No buffer needs a "free" signal.  A peer sends tile i + kBuf's data only after its phase A of that
+        // tile has completed, hence (its MMAs run in order) after its phase C of tile i, hence after it has
+        // received my tile-i sums, which I sent after reading the tile-i contributions.  And the T operand
+        // buffer of a receiver is free once its phase A of tile i is complete (phase C of tile i - kBuf was
+        // issued before it), which is before it sends the contribution that my sum of tile i waits for.
+        float* rs = sRs + p * kRsFloats;          // [C sources][cpo groups][8 tokens][NP]
+        const int my_c = (kTT / 8 - rank + C - 1) / C;      // token groups of a tile that this CTA owns
         if (et == 0) {
-          mbar_expect_tx(&sh.rs_full[p], (uint32_t)(C * my_rows * NP * 4));
-          mbar_expect_tx(&sh.ag_full[p], (uint32_t)(kTT * NP * 4));
+          mbar_expect_tx(&sh.rs_full[p], (uint32_t)(C * my_c * 8 * NP * 4));
+          mbar_expect_tx(&sh.tt_full[p], (uint32_t)(NP * kTT * 4));
         }
         if (lane < 16) {
-          const int R = 16 * q + lane, dest = R / rows_per, lrow = R - dest * rows_per;
-          const uint32_t dst = mapa_shared(smem_u32(rs + (rank * rows_per + lrow) * NP), (uint32_t)dest);
+          const int R = 16 * q + lane, j = R >> 3, dest = j % C, jc = j / C;
+          const uint32_t dst = mapa_shared(smem_u32(rs + ((rank * cpo + jc) * 8 + (R & 7)) * NP), (uint32_t)dest);
           const uint32_t bar = mapa_shared(smem_u32(&sh.rs_full[p]), (uint32_t)dest);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
@@ -307,53 +325,40 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         ok = mbar_wait_cluster(&sh.rs_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
+        // Every warp of the group adds the C contributions of an owned token group (lane = (token of the
+        // group, four rank indices); the four warps do the same additions, which is cheaper than handing
+        // the sums over), passes the bf16 parts through its 512-byte staging block so that a lane then
+        // holds one 16-byte piece (eight tokens of one operand row), and sends it to the CTAs d = q mod 4.
         {
-          const int q4 = NP >> 2;                 // float4 pieces per row
-          for (int u = et; u < my_rows * q4; u += 128) {
-            const int lrow = u / q4, k4 = u - lrow * q4;
-            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int c = 0; c < C; ++c) {
-              const float4 v = *reinterpret_cast<const float4*>(rs + (c * rows_per + lrow) * NP + 4 * k4);
-              sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+          __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(sStage) + ((grp * 4 + q) * 32 * 8);
+          const uint32_t tt_base = smem_u32(sTt) + (uint32_t)p * 32u * 128u;
+          const uint32_t tt_bar = smem_u32(&sh.tt_full[p]);
+          for (int jc = 0; jc < my_c; ++jc) {
+            const int x = lane & 7, kq = lane >> 3;
+            if (4 * kq < NP) {
+              float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+              for (int c = 0; c < C; ++c) {
+                const float4 v = *reinterpret_cast<const float4*>(rs + ((c * cpo + jc) * 8 + x) * NP + 4 * kq);
+                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+              }
+              const float sv[4] = {sum.x, sum.y, sum.z, sum.w};
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(sv[c]);
+                stage[(4 * kq + c) * 8 + x] = h;
+                stage[(NP + 4 * kq + c) * 8 + x] = __float2bfloat16_rn(sv[c] - __bfloat162float(h));
+              }
             }
-            const uint32_t off = smem_u32(ag + (rank * rows_per + lrow) * NP + 4 * k4);
-            const uint32_t bar = smem_u32(&sh.ag_full[p]);
-            for (int c = 0; c < C; ++c) st_async_f4(mapa_shared(off, (uint32_t)c), sum, mapa_shared(bar, (uint32_t)c));
+            __syncwarp();
+            if (lane < 2 * NP) {      // operand rows: hi parts 0..NP-1, then lo parts
+              const uint4 piece = *reinterpret_cast<const uint4*>(stage + lane * 8);
+              const uint32_t pv[4] = {piece.x, piece.y, piece.z, piece.w};
+              const uint32_t off = tt_base + swz(lane, rank + C * jc);
+              for (int d = q; d < C; d += 4) st_async_u4(mapa_shared(off, (uint32_t)d), pv, mapa_shared(tt_bar, (uint32_t)d));
+            }
+            __syncwarp();
           }
         }
-        ok = mbar_wait_cluster(&sh.ag_full[p], u2 & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        // thread = (token row, half of the NP values of T)
-        const int row = 16 * q + (lane & 15), kh = (lane >> 4) * hn;
-        float acc[8];
-        {
-          const float4 a = *reinterpret_cast<const float4*>(ag + row * NP + kh);
-          acc[0] = a.x; acc[1] = a.y; acc[2] = a.z; acc[3] = a.w;
-          float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (hn == 8) b = *reinterpret_cast<const float4*>(ag + row * NP + kh + 4);
-          acc[4] = b.x; acc[5] = b.y; acc[6] = b.z; acc[7] = b.w;
-        }
-        // T operand of phase C: rows = hi parts 0..NP-1 then lo parts, 64 tokens (128 bytes) per row
-        if (u2 > 0) {
-          ok = mbar_wait(&sh.tt_empty[p], (u2 - 1) & 1);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
-        uint8_t* tt = sTt + (size_t)p * 32 * 128;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (j >= hn) break;
-          const float v = acc[j];
-          const __nv_bfloat16 h = __float2bfloat16_rn(v);
-          const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
-          const int k = kh + j;
-          *reinterpret_cast<__nv_bfloat16*>(tt + swz(k, row >> 3) + (row & 7) * 2) = h;
-          *reinterpret_cast<__nv_bfloat16*>(tt + swz(NP + k, row >> 3) + (row & 7) * 2) = l;
-        }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.tt_full[p]);
       }
       if (!ok) break;
       if (grp != 0) continue;
@@ -392,9 +397,9 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
 int g_max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // per cluster size, filled on first use
 
 size_t fz_smem_bytes(int ring) {
-  return (size_t)ring * kSlotBytes + 8 * 32 * 128 + 2 * 32 * 128 + 2 * kRsFloats * 4 + 2 * kTT * 16 * 4 + 1024;
+  return (size_t)ring * kSlotBytes + 8 * 32 * 128 + kBuf * 32 * 128 + kBuf * kRsFloats * 4 + 8 * 512 + 1024;
 }
-constexpr int kFzRing = 10;
+constexpr int kFzRing = 10;    // as many slots as fit beside the other regions in 227 KiB
 
 }  // namespace
 
@@ -442,7 +447,9 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   cfg.gridDim = dim3((unsigned)(nclusters * C));
   const DevLayer* layers = w.d_layers;
   int l0 = w.l0, l1 = w.l1, ring = kFzRing;
-  void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&ring, (void*)&d_status};
+  int pf = 4;
+  if (const char* e = getenv("AGZO_FZ_PF")) pf = atoi(e);
+  void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&ring, (void*)&pf, (void*)&d_status};
   return cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel, args);
 }
 
