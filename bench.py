@@ -133,17 +133,45 @@ def algorithmic_work(cfg: WL.LayerSetConfig, rank: int, alias_inputs: bool = Fal
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
-def oracle_block_seconds(cfg: WL.LayerSetConfig, rank: int, X_host, W_host, seed: int = 0):
-    """The oracle, as it stands, on block 0 (7 layers): Algorithm 1 + the three passes."""
+def oracle_layer_seconds(cfg: WL.LayerSetConfig, rank: int, X_host, W_host, seed: int = 0):
+    """The oracle, as it stands, on the given layers (Algorithm 1 + the three passes of a two-point
+    step); returns the seconds each layer took."""
     from oracle import agzo_oracle as O
-    t0 = time.perf_counter()
+    out = []
     for i, (X, W) in enumerate(zip(X_host, W_host)):
+        t0 = time.perf_counter()
         V = O.extract_subspace(X, rank, K_POWER, seed, i)
         W1 = O.apply_direction(W, V, seed, i, np.float32(EPS), "bf16")
         W2 = O.apply_direction(W1, V, seed, i, np.float32(-2 * EPS), "bf16")
         g = O.ghat_two_point(1.0, 0.999, EPS)
         O.apply_direction(W2, V, seed, i, O.update_coefficient(EPS, LR, g, 0), "bf16")
-    return time.perf_counter() - t0
+        out.append(time.perf_counter() - t0)
+    return out
+
+
+def oracle_block_seconds(cfg: WL.LayerSetConfig, rank: int, X_host, W_host, seed: int = 0):
+    """Block 0 (7 layers) through the oracle: the sample both CPU legs time."""
+    return float(sum(oracle_layer_seconds(cfg, rank, X_host, W_host, seed)))
+
+
+def cpu_baseline_leg(cfg: WL.LayerSetConfig, rank: int, n_layers_total: int):
+    """The oracle on block 0 with all host cores (every block has the same shapes, so the block's time
+    is multiplied by the number of blocks), and its second layer once more on one thread."""
+    Xh, Wh = host_block(cfg)
+    per_layer = oracle_layer_seconds(cfg, rank, Xh, Wh)
+    t = float(sum(per_layer))
+    out = {"value": t * 1e3 * cfg.n_blocks, "unit": "ms", "cores": os.cpu_count(), "kind": "oracle",
+           "sample": f"block 0 ({len(cfg.block)} of {n_layers_total} layers) timed ({t:.1f} s), "
+                     f"time x{cfg.n_blocks} blocks"}
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            t1 = oracle_layer_seconds(cfg, rank, Xh[1:2], Wh[1:2])[0]
+        out["single_thread"] = {"sample": "layer 1 of block 0 (%s)" % cfg.block[1][0], "seconds_one_thread": t1,
+                                "seconds_all_cores": per_layer[1]}
+    except Exception as e:  # noqa: BLE001 - the thread limit is a convenience of the report
+        out["single_thread"] = {"unavailable": repr(e)}
+    return out
 
 
 def host_block(cfg: WL.LayerSetConfig, n_layers: int = 7, seed: int = 1000):
@@ -155,34 +183,68 @@ def host_block(cfg: WL.LayerSetConfig, n_layers: int = 7, seed: int = 1000):
     return Xs, Ws
 
 
+def workload_string(cfg: WL.LayerSetConfig, rank_r: int, mode: int) -> str:
+    """The one description of the workload that both arms print."""
+    return (f"{cfg.name}: {len(cfg.layers())} layers, {cfg.n_params() / 1e9:.3f} G weights, m={cfg.m} tokens, "
+            f"r={rank_r}, K={K_POWER}, eps={EPS}, " + ("two-point" if mode == 0 else "one-sided"))
+
+
 def run_reference(args, cfg, rank_r):
     """--impl reference: the CPU oracle on the host cores; a step = block 0 of the layer set,
     extrapolated to all blocks (every block has the same shapes)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return 0
     cores = os.cpu_count() or 1
-    # a step is bounded so that the whole run ends within a few minutes: the whole block for short
-    # runs, its first two layers for long ones, scaled by the elements a layer touches
-    n_sample = len(cfg.block) if args.warmup + args.steps <= 8 else 2
-    Xs, Ws = host_block(cfg, n_sample)
-    touched = lambda layers: sum(di * (cfg.m + do) for (_, di, do) in layers)
-    scale = touched(cfg.block) / touched(cfg.block[:n_sample])
-    times = []
-    for it in range(args.warmup + args.steps):
-        t = oracle_block_seconds(cfg, rank_r, Xs, Ws, seed=it)
+    # A step is the sample the cpu_baseline leg of the main arm times: block 0, whole.  The first
+    # step always runs it whole; if all W + K steps at that pace would take more than about four
+    # minutes, the later steps time the block's first two layers and are scaled by the ratio that
+    # the first step measured between the whole block and those two layers.
+    Xs, Ws = host_block(cfg)
+    total = args.warmup + args.steps
+    first = oracle_layer_seconds(cfg, rank_r, Xs, Ws, seed=0)
+    t_block, t_two = float(sum(first)), float(sum(first[:2]))
+    whole = t_block * total <= 240.0
+    scale = 1.0 if whole else t_block / t_two
+    times = [t_block] if args.warmup == 0 else []
+    for it in range(1, total):
+        t = (oracle_block_seconds(cfg, rank_r, Xs, Ws, seed=it) if whole
+             else float(sum(oracle_layer_seconds(cfg, rank_r, Xs[:2], Ws[:2], seed=it))) * scale)
         if it >= args.warmup:
             times.append(t)
-    ms = float(np.mean(times)) * 1e3 * scale * cfg.n_blocks
-    sample = (f"first {n_sample} of the {len(cfg.block)} layers of block 0 per step, time x{scale:.2f} "
-              f"(elements touched) x{cfg.n_blocks} blocks")
+    ms = float(np.mean(times)) * 1e3 * cfg.n_blocks
+    sample = (f"block 0 ({len(cfg.block)} layers) per step, time x{cfg.n_blocks} blocks" if whole else
+              f"block 0 whole in the first step ({t_block:.1f} s); later steps its first 2 layers x{scale:.2f} "
+              f"(ratio measured in the first step), time x{cfg.n_blocks} blocks")
     line = {"metric": METRIC, "value": ms, "unit": "ms", "impl": "reference", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}, r={rank_r}, K={K_POWER}, m={cfg.m}", "sample": sample},
+            "config": {"workload": workload_string(cfg, rank_r, 0), "sample": sample},
             "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": ms, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
     return 0
+
+
+def spawn_ranks(n: int, argv, worker=None, env_extra=None, port: int | None = None):
+    """Starts n local processes, one per GPU, as a launcher would: RANK / LOCAL_RANK / WORLD_SIZE /
+    MASTER_ADDR / MASTER_PORT in the environment, the same command line.  `worker` replaces
+    [python, bench.py] (the tests pass a stub).  Returns the exit codes in rank order."""
+    import socket
+    if port is None:
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+    cmd = list(worker) if worker is not None else [sys.executable, os.path.abspath(__file__)]
+    procs = []
+    for rk in range(n):
+        env = dict(os.environ)
+        env.update({"RANK": str(rk), "LOCAL_RANK": str(rk), "WORLD_SIZE": str(n), "LOCAL_WORLD_SIZE": str(n),
+                    "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+        env.setdefault("NCCL_DEBUG", "INFO" if rk == 0 else "WARN")     # the communicator's own log stays on
+        if env_extra:
+            env.update(env_extra)
+        procs.append(subprocess.Popen(cmd + list(argv), env=env))
+    return [p.wait() for p in procs]
 
 
 def max_over_ranks(ms: float, dist, device) -> float:
@@ -197,6 +259,76 @@ def max_over_ranks(ms: float, dist, device) -> float:
 def whole_job_units(per_rank_units: float, world: int) -> float:
     """Replicas (weak scaling): every rank does the same per-rank work, the job does world times it."""
     return per_rank_units * world
+
+
+# ----------------------------------------------------------------------------- sweep
+def sweep_entry(B, cfg, r, Ws, Xs, dev, local, peak, steps=3, wave_bytes=None, label=None):
+    """One short run of the whole step on a resident layer set at rank r: step, extraction and one
+    pass (CUDA events), the pass's bandwidth, the device status."""
+    Vs = [torch.zeros(r, X.shape[1], dtype=torch.float32, device=dev) for X in Xs]
+    layers = [B.make_layer(W=W, X=X, V=V, r=r, layer_id=i) for i, (W, X, V) in enumerate(zip(Ws, Xs, Vs))]
+    arr = B.layer_array(layers)
+    ctx = B.agzo_create(layers, local)
+    if wave_bytes is not None:
+        B.agzo_set_option(ctx, "wave_bytes", wave_bytes)
+    losses = torch.tensor([1.0, 0.999], dtype=torch.float64, device=dev)
+    ghat = torch.zeros(1, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(seed):
+        B.agzo_extract_subspace(ctx, layers, seed, K_POWER, arr=arr)
+        B.agzo_perturb(ctx, layers, seed, EPS, arr=arr)
+        B.agzo_perturb(ctx, layers, seed, -2 * EPS, arr=arr)
+        B.agzo_ghat(ctx, losses[0:1], losses[1:2], EPS, 0, ghat)
+        B.agzo_restore_update(ctx, layers, seed, EPS, LR, 0, ghat, arr=arr)
+
+    def ms_of(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(n):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    step(0); step(1); step(2)          # warm-up
+    ms_step = ms_of(lambda i: step(10 + i), steps)
+    ms_extract = ms_of(lambda i: B.agzo_extract_subspace(ctx, layers, 200 + i, K_POWER, arr=arr), 2)
+    ms_pass = ms_of(lambda i: B.agzo_perturb(ctx, layers, 300 + i, EPS if i % 2 == 0 else -EPS, arr=arr), 4)
+    status = B.agzo_poll(ctx)
+    B.agzo_destroy(ctx)
+    work = algorithmic_work(cfg, r)
+    gbps = work["rmw_bytes_per_pass"] / ms_pass / 1e6
+    return {"workload": label or cfg.name, "r": r, "step_ms": ms_step, "extract_ms": ms_extract, "pass_ms": ms_pass,
+            "pass_GBps": gbps, "pass_frac_of_measured_hbm": gbps / peak, "pass_frac_of_nominal_8TBps": gbps / 8000.0,
+            "extract_GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6,
+            "device_status": B.status_string(status)}
+
+
+def run_sweep(B, args, cfg_head, Ws, Xs, dev, local, peak):
+    """The rest of the measurement grid, a few steps each: the other ranks of the headline layer set,
+    then the 1.7B- and 0.6B-shaped sets (the big set is freed first).  For the 0.6B-shaped set, whose
+    activation matrices (17 to 50 MB) fit L2, extraction is also timed in waves of one or two layers,
+    so that the seven sweeps over a layer's X after the first find it in L2."""
+    out = []
+    for r in (1, 4, 64):
+        if r != args.rank:
+            out.append(sweep_entry(B, cfg_head, r, Ws, Xs, dev, local, peak))
+    Ws.clear(); Xs.clear()
+    torch.cuda.empty_cache()
+    for cfg, ranks in ((WL.QWEN3_1P7B, (4, 8, 16)), (WL.QWEN3_0P6B, (8,))):
+        W2, X2, _, _ = build_layer_set(cfg, 1, dev)
+        for r in ranks:
+            out.append(sweep_entry(B, cfg, r, W2, X2, dev, local, peak))
+        if cfg is WL.QWEN3_0P6B:
+            e = sweep_entry(B, cfg, 8, W2, X2, dev, local, peak, wave_bytes=56 << 20,
+                            label=cfg.name + ", extraction in waves of at most 56 MB of activations (X stays in L2 "
+                                             "across the sweeps of a wave)")
+            out.append(e)
+        del W2, X2
+        torch.cuda.empty_cache()
+    return out
 
 
 # ----------------------------------------------------------------------------- main arm
@@ -233,6 +365,8 @@ def main():
                     help="every rank's activations are its own tokens of one batch of N x m tokens: extraction sums "
                          "the Y panels over the ranks (NCCL all-reduce through agzo_set_allreduce); the in-place "
                          "passes stay replicated.  Default: independent replicas")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the short sweep over the other ranks and layer sets that follows the headline region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -244,6 +378,12 @@ def main():
     r = args.rank
     if args.impl == "reference":
         return run_reference(args, cfg, r)
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        # started as a plain command: be the launcher (one process per GPU, NCCL over 127.0.0.1)
+        if not torch.cuda.is_available() or torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus}: {torch.cuda.device_count() if torch.cuda.is_available() else 0} "
+                             "CUDA devices visible")
+        return max(spawn_ranks(args.gpus, sys.argv[1:]))
 
     from paper_2601_17261_b200 import binding as B
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -396,8 +536,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic",
             "data": "synthetic", "method": args.method,
-            "config": {"workload": f"{cfg.name}: {len(layers)} layers, {cfg.n_params() / 1e9:.3f} G weights, "
-                                   f"m={cfg.m} tokens, r={r}, K={K_POWER}, eps={EPS}, " + ("two-point" if args.mode == 0 else "one-sided"),
+            "config": {"workload": workload_string(cfg, r, args.mode),
                        "l2": "inputs larger than L2 (weights %.1f GB + activations %.1f GB per step)"
                              % (work["w_bytes"] / 1e9, work["x_bytes"] / 1e9),
                        "replicas": world, "device_status": B.status_string(status),
@@ -414,7 +553,10 @@ def main():
                         "GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6},
             "roofline": {"kernel": ("tc_xt_t_kernel" if tc_used else "xt_t_kernel") + " (Y = X^T T)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+                         "frac_of_nominal_8TBps": (achieved / 8000.0) if achieved else None,
                          "peak_kind": peak_kind,
+                         "peak_note": "the peak is the copy rate measured on this pool (a read-and-write stream): a "
+                                      "reference rate, not a ceiling -- a read-only sweep can exceed it",
                          "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE["tc_xt_t_kernel"] * x_bytes_per_launch
                                      if tc_used and dom_n else None),
                          "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the "
@@ -427,15 +569,16 @@ def main():
         if e2e:
             line["e2e"] = e2e
         if not args.no_cpu_baseline and world == 1:
-            Xh, Wh = host_block(cfg)
             # one transformer block (every block has the same shapes): tens of seconds of CPU work
-            t = oracle_block_seconds(cfg, r, Xh, Wh)
-            line["cpu_baseline"] = {"value": t * 1e3 * cfg.n_blocks, "unit": "ms",
-                                    "cores": os.cpu_count(), "kind": "oracle",
-                                    "sample": f"block 0 ({len(cfg.block)} of {len(layers)} layers) timed ({t:.1f} s), "
-                                              f"time x{cfg.n_blocks} blocks"}
-        print(json.dumps(line))
+            line["cpu_baseline"] = cpu_baseline_leg(cfg, r, len(layers))
     B.agzo_destroy(ctx)
+    ctx.workspace = None          # the sweep below sizes its own workspaces
+    if rank == 0:
+        if (not args.no_sweep and world == 1 and args.method == "agzo" and args.mode == 0 and args.blocks == 0
+                and cfg is WL.QWEN3_8B and not args.alias_inputs):
+            del layers, arr, Vs
+            line["sweep"] = run_sweep(B, args, cfg, Ws, Xs, dev, local, peak)
+        print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
     return 0

@@ -105,3 +105,23 @@ def test_reference_arm_runs_on_rank_zero_only():
                         "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert p.returncode == 0
     assert not [l for l in p.stdout.splitlines() if l.startswith("{")]
+
+
+def test_bench_launcher_starts_one_process_per_rank(tmp_path):
+    """`python bench.py --gpus N` run as a plain command starts N local ranks itself.  The launcher is
+    exercised here with a stub worker: every process must see its own RANK / LOCAL_RANK, the common
+    WORLD_SIZE and a rendezvous on 127.0.0.1, and the exit codes come back in rank order."""
+    import bench
+    stub = ("import os, sys; d = sys.argv[1]; r = os.environ['RANK']; "
+            "open(os.path.join(d, 'rank_' + r), 'w').write(' '.join(os.environ[k] for k in "
+            "('RANK', 'LOCAL_RANK', 'WORLD_SIZE', 'MASTER_ADDR', 'MASTER_PORT'))); sys.exit(3 if r == '2' else 0)")
+    codes = bench.spawn_ranks(4, [str(tmp_path)], worker=[sys.executable, "-c", stub])
+    assert codes == [0, 0, 3, 0]
+    seen = sorted(p.name for p in tmp_path.iterdir())
+    assert seen == ["rank_0", "rank_1", "rank_2", "rank_3"]
+    ports = set()
+    for i in range(4):
+        rank, local, world, addr, port = (tmp_path / f"rank_{i}").read_text().split()
+        assert (rank, local, world, addr) == (str(i), str(i), "4", "127.0.0.1")
+        ports.add(port)
+    assert len(ports) == 1
