@@ -108,3 +108,120 @@ def test_agzo_steps_on_a_transformer_block(dtype, r):
             assert ratios and all(0.7 <= x <= 1.3 for x in ratios), ratios
     finally:
         B.agzo_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------------
+# Algorithm 2, step 1 as printed: "obtain H_l using hooks ... A_l <- SubspaceExtract(H_l, r_l, K)" during
+# the unperturbed forward, after which H_l is discarded.  One Qwen3-8B-shaped block (hidden 4096, 32 query /
+# 8 key-value heads of 128, intermediate 12288) on 8 x 2048 tokens in bf16: forward pre-hooks hand the input
+# of each group of linear layers (q/k/v, o, gate/up, down) to the library on the forward's stream, right
+# after the op that produced it; the activation tensor is torch's temporary and is never kept.
+class _QwenBlock(torch.nn.Module):
+    def __init__(self, hid=4096, heads=32, kv_heads=8, head_dim=128, inter=12288, seed=0):
+        super().__init__()
+        self.heads, self.kv_heads, self.head_dim = heads, kv_heads, head_dim
+        g = torch.Generator(device="cpu").manual_seed(seed)
+
+        def lin(d_in, d_out):
+            layer = torch.nn.Linear(d_in, d_out, bias=False, device=DEV, dtype=torch.bfloat16)
+            with torch.no_grad():
+                layer.weight.copy_((torch.randn(d_out, d_in, generator=g) * 0.02).to(torch.bfloat16))
+            return layer
+
+        self.q, self.k, self.v = lin(hid, heads * head_dim), lin(hid, kv_heads * head_dim), lin(hid, kv_heads * head_dim)
+        self.o = lin(heads * head_dim, hid)
+        self.gate, self.up, self.down = lin(hid, inter), lin(hid, inter), lin(inter, hid)
+
+    @staticmethod
+    def _norm(x):
+        xf = x.float()
+        return (xf * torch.rsqrt((xf * xf).mean(-1, keepdim=True) + 1e-6)).to(x.dtype)
+
+    def forward(self, x):
+        b, t, _ = x.shape
+        h = self._norm(x)
+        q = self.q(h).view(b, t, self.heads, self.head_dim).transpose(1, 2)
+        k = self.k(h).view(b, t, self.kv_heads, self.head_dim).transpose(1, 2)
+        v = self.v(h).view(b, t, self.kv_heads, self.head_dim).transpose(1, 2)
+        rep = self.heads // self.kv_heads
+        a = torch.nn.functional.scaled_dot_product_attention(q, k.repeat_interleave(rep, 1), v.repeat_interleave(rep, 1),
+                                                             is_causal=True)
+        x = x + self.o(a.transpose(1, 2).reshape(b, t, -1))
+        h2 = self._norm(x)
+        return x + self.down(torch.nn.functional.silu(self.gate(h2)) * self.up(h2))
+
+
+def test_extraction_inside_the_forward_of_an_8b_shaped_block():
+    from oracle import agzo_oracle as O
+    from gpu_helpers import projector_distance, to_host
+    torch.cuda.empty_cache()
+    if torch.cuda.mem_get_info()[0] < 24 * 2 ** 30:
+        pytest.skip("needs 24 GB of free device memory")
+    r, K, seed, batch, seq = 16, 3, 17, 8, 2048
+    blk = _QwenBlock()
+    groups = {"q": ["q", "k", "v"], "o": ["o"], "gate": ["gate", "up"], "down": ["down"]}
+    order = ["q", "k", "v", "o", "gate", "up", "down"]
+    mods = {n: getattr(blk, n) for n in order}
+    Vs = {n: torch.zeros(r, mods[n].in_features, device=DEV) for n in order}
+    m = batch * seq
+
+    def descriptors(names, X):
+        return [B.make_layer(W=mods[n].weight, X=X, V=Vs[n], r=r, layer_id=order.index(n)) for n in names]
+
+    # workspace for the largest call: all seven layers at once (the X pointer only has to be non-null here)
+    sizing = [B.make_layer(W=mods[n].weight, X=mods[n].weight, V=Vs[n], r=r, layer_id=i) for i, n in enumerate(order)]
+    for L, n in zip(sizing, order):
+        L.m, L.ldx = m, mods[n].in_features
+    ctx = B.agzo_create(sizing, 0)
+    host_X, hooked_ms, events = {}, [], []
+
+    def make_hook(first):
+        def hook(module, args):
+            X = args[0].reshape(-1, args[0].shape[-1])           # [tokens][d_in] view of torch's temporary
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.agzo_extract_subspace(ctx, descriptors(groups[first], X), seed, K)
+            e1.record()
+            events.append((e0, e1))
+            host_X[first] = X.float().cpu().numpy()              # the test's copy for the oracle; the library keeps nothing
+        return hook
+
+    handles = [mods[first].register_forward_pre_hook(make_hook(first)) for first in groups]
+    try:
+        g = torch.Generator(device="cpu").manual_seed(5)
+        x0 = torch.randn(batch, seq, 4096, generator=g).to(DEV).to(torch.bfloat16)
+        with torch.no_grad():
+            out = blk(x0)
+        torch.cuda.synchronize()
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+        assert bool(torch.isfinite(out.float()).all())
+        hooked = sum(a.elapsed_time(b) for a, b in events)
+    finally:
+        for h in handles:
+            h.remove()
+    # every layer's basis against the oracle on the same activations
+    for first, names in groups.items():
+        for n in names:
+            Vg = to_host(Vs[n])
+            Vo = O.extract_subspace(host_X[first], r, K, seed, order.index(n))
+            assert np.abs(Vg.astype(np.float64) @ Vg.T - np.eye(r)).max() <= 1e-5, n
+            assert projector_distance(Vg, Vo) <= 1e-3, n
+    # the same extraction from resident buffers, one call over all seven layers (shared inputs grouped)
+    Xres = {first: torch.from_numpy(host_X[first]).to(DEV).to(torch.bfloat16) for first in groups}
+    first_of = {n: first for first, names in groups.items() for n in names}
+    layers = [B.make_layer(W=mods[n].weight, X=Xres[first_of[n]], V=Vs[n], r=r, layer_id=i) for i, n in enumerate(order)]
+    B.agzo_extract_subspace(ctx, layers, seed, K)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    B.agzo_extract_subspace(ctx, layers, seed, K)
+    e1.record()
+    torch.cuda.synchronize()
+    resident = e0.elapsed_time(e1)
+    assert B.agzo_poll(ctx) == B.AGZO_OK
+    B.agzo_destroy(ctx)
+    print(f"\nextraction of one 8B-shaped block, r = {r}: {hooked:.3f} ms inside the forward (four hook calls, "
+          f"activations just written), {resident:.3f} ms from resident buffers in one call")
+    # the hooked form serves one group per call and cannot overlap the groups' panel QR with other sweeps;
+    # it must stay in the same range
+    assert hooked <= 2.0 * resident + 1.0
