@@ -35,6 +35,9 @@ K_POWER = 3
 # slice of the 8B-shaped layer set (summaries under profiles/); traffic grows in proportion
 # to the activation bytes a launch sweeps.  Reset an entry to None when its kernel changes.
 TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (4.865842 + 0.012305) / 4.831838}
+# Thread-level instructions per weight of the dense-direction kernel (one Philox + Box-Muller normal per weight):
+# ncu smsp__thread_inst_executed.sum / weights on a 4096 x 4096 bf16 layer (profiles/dense_vec_kernel_*.md).
+DENSE_INST_PER_WEIGHT = 933126144 / (4096 * 4096)
 EPS = 1e-3
 LR = 1e-6
 METRIC = "agzo_step_overhead_ms"
@@ -566,6 +569,19 @@ def main():
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
+        if args.method == "mezo":
+            # the dense pass is bound by the arithmetic of its normals: instructions issued per second against
+            # what the SMs can issue (4 schedulers x 32 lanes per SM and clock)
+            sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+            mhz = clocks.get("sm_max_mhz") or 1965.0
+            peak_alu = sm_count * 128 * mhz * 1e6 / 1e12
+            ach = cfg.n_params() * DENSE_INST_PER_WEIGHT / (ms_step / 3 * 1e-3) / 1e12
+            line["roofline"] = {"kernel": "dense_vec_kernel (w += c u, u ~ N(0, I) from the counter)", "bound": "alu",
+                                "achieved": ach, "peak": peak_alu, "unit": "T thread-instructions/s",
+                                "frac": ach / peak_alu, "traffic": None, "ms_per_pass": ms_step / 3,
+                                "inst_per_weight": DENSE_INST_PER_WEIGHT,
+                                "peak_note": "SMs x 128 lanes x the maximum SM clock; instructions per weight from ncu",
+                                "GBps": 4 * cfg.n_params() / (ms_step / 3) / 1e6}
         if e2e:
             line["e2e"] = e2e
         if not args.no_cpu_baseline and world == 1:

@@ -248,6 +248,34 @@ def test_dense_direction():
         assert d.max() <= 1 and (d > 0).mean() < 1e-3
 
 
+@pytest.mark.parametrize("n,bf16,offset", [(100003, False, 0), (4099, True, 1), (4099, False, 3), (5, True, 0), (8, True, 0),
+                                             (1 << 20, True, 0)])
+def test_dense_direction_sizes_dtypes_and_alignments(n, bf16, offset):
+    # vector path (16-byte aligned, eight elements per thread) with its scalar tail, the scalar path for a
+    # vector that does not start on a 16-byte boundary, fp32 storage, tiny vectors; sentinels on both sides
+    w0 = WL.gaussian_weights(1, n, 0.5, seed=n + offset, bf16=bf16).reshape(-1)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    buf = torch.full((n + offset + 16,), 7.0, dtype=dt, device=DEV)
+    wd = buf[offset:offset + n]
+    wd.copy_(torch.from_numpy(w0).to(DEV).to(dt))
+    V = torch.zeros(1, 8, device=DEV)
+    with Ctx([B.make_layer(V=V, r=1, layer_id=0, d_in=8)]) as ctx:
+        B.agzo_perturb_dense(ctx, wd, 6, 35, 3e-2)
+        torch.cuda.synchronize()
+    want = O.apply_dense(w0, 6, 35, np.float32(3e-2), "bf16" if bf16 else "f32")
+    got = to_host(wd)
+    if bf16:
+        d = bf16_ulp_distance(got, want)
+        assert d.max() <= 1 and (d > 0).mean() < 1e-3 + 2.0 / n
+    else:
+        # 4 fp32 ulp of the operands: where w + c u cancels, the result's own ulp is below the rounding of the
+        # normals (a few 1e-7 relative), which no fp32 evaluation can beat
+        u = np.abs(O.gen_dense(6, 35, n).astype(np.float64))
+        scale = np.maximum(np.abs(w0.astype(np.float64)), 3e-2 * u)
+        assert np.all(np.abs(got.astype(np.float64) - want) <= 4 * 2.0 ** -23 * scale)
+    assert bool((buf[:offset] == 7).all() and (buf[offset + n:] == 7).all())
+
+
 def test_gaussian_right_factor_matches_the_oracle_and_feeds_the_passes():
     specs = [(300, 640, 8), (64, 100, 3)]
     devs, layers = [], []
