@@ -155,7 +155,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
           const int t0 = it.t_begin + tile * kTT;
           for (int b = 0; b < mb; ++b, ++ns) {
             const int s = ns % ring, u = ns / ring;
-            if (u > 0 && !mbar_wait_spin(&sh.x_empty[s], (u - 1) & 1)) { ok = false; break; }
+            if (u > 0 && !mbar_wait(&sh.x_empty[s], (u - 1) & 1)) { ok = false; break; }
             uint8_t* slot = sX + (size_t)s * kSlotBytes;
             mbar_expect_tx(&sh.x_full[s], kSlotBytes);
             tma_load_2d(slot, map_x, col0 + 128 * b, t0, &sh.x_full[s]);
@@ -269,7 +269,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       for (int tile = 0; tile < it.ntiles && ok; ++tile, ++te) {
         const int p = te % kBuf, u2 = te / kBuf;
         if ((te & 1) != grp) continue;
-        ok = mbar_wait_spin(&sh.tp_full[p], u2 & 1);
+        ok = mbar_wait(&sh.tp_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();

@@ -61,18 +61,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     if (global_ns() - t0 > kWaitCapNs) return false;
   }
 }
-// Bounded wait that polls instead of suspending: for waits on the critical path of a pipeline,
-// where the wake-up of a suspended thread would add to every hand-over.
-__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > kWaitCapNs) return false;
-  }
-}
 __device__ __forceinline__ void tma_load_2d(void* dst, const void* tmap, int c0, int c1, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -179,7 +167,7 @@ __device__ __forceinline__ void mma_commit_if(uint32_t go, uint64_t* bar) {
 }
 // bounded wait by a whole warp; the answer is made the same for all lanes
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity) {
-  const bool ok = mbar_wait_spin(bar, parity);
+  const bool ok = mbar_wait(bar, parity);
   return __all_sync(0xffffffffu, ok);
 }
 
@@ -254,19 +242,21 @@ __device__ __forceinline__ uint32_t cluster_count_x() {
 __device__ __forceinline__ uint32_t mapa_shared(uint32_t saddr, uint32_t rank) {
   uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank)); return r;
 }
-// bounded wait with acquire at cluster scope: for barriers that CTAs of the cluster arrive on
+// bounded wait with acquire at cluster scope: for barriers that CTAs of the cluster arrive on.  The thread
+// suspends inside try_wait (the hardware wakes it when the phase completes): hundreds of threads polling a
+// barrier keep the shared-memory pipeline busy that the arrivals themselves have to pass through.
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {
   const unsigned long long t0 = global_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 64; ++i) {
+    for (int i = 0; i < 16; ++i) {
       uint32_t ok;
       asm volatile(
           "{\n\t.reg .pred p;\n\t"
-          "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+          "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
           "selp.u32 %0, 1, 0, p;\n\t}"
           : "=r"(ok)
-          : "r"(smem_u32(bar)), "r"(parity)
+          : "r"(smem_u32(bar)), "r"(parity), "r"(4000u)
           : "memory");
       if (ok) return true;
     }
