@@ -23,7 +23,10 @@
  *     that uses it is in flight.  The library keeps no other pointer past a call.
  *   - All work is enqueued on the caller's stream (a cudaStream_t passed as void*) and the
  *     calls return without waiting for it, except where stated.  Calls that share a context
- *     must be issued on one stream or be ordered by the caller.
+ *     must be issued on one stream or be ordered by the caller (they share the workspace).
+ *     Two pieces of state the library itself carries from call to call are made safe across a
+ *     change of stream: the new stream waits for the last upload of the layer tables, and
+ *     staged R operand images written on another stream are rewritten instead of reused.
  *   - Every function returns an agzo_status; nothing throws, traps or aborts.  Argument
  *     errors are detected on the host before anything is launched.  Conditions that only
  *     the device can see (a rank-deficient panel, a wait that ran out) are written to a
