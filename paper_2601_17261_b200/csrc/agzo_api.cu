@@ -193,7 +193,7 @@ void slab_shape(const agzo_layer& a, bool tc, bool long_slabs, int* slabs, int* 
   int rows;
   if (tc) {
     rows = a.m >= 8192 ? (long_slabs ? (a.m < 16384 ? a.m : 16384) : 2048) : (a.m + 3) / 4;
-    rows = (rows + 63) / 64 * 64;
+    rows = (rows + 127) / 128 * 128;      // whole tiles of every tensor-core kernel (64 or 128 tokens)
   } else {
     rows = (a.m + 31) / 32;
     rows = (rows + 31) / 32 * 32;

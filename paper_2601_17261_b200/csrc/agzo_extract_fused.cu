@@ -1,38 +1,34 @@
-// One power step of Algorithm 1, Y <- H (H^T Q) = X^T (X Q), in a single pass over X.
+// One power step of Algorithm 1, Y <- H (H^T Q) = X^T (X Q), with X crossing HBM once.
 //
 // The two products of a power step meet the same X: T = X Q needs a whole row of X (all of d_in)
-// before a single element of Y = X^T T can be formed, so the unfused kernels read X twice.  Here a
-// thread-block cluster of C CTAs shares a tile of 64 tokens; CTA c keeps its 512-column slice of
-// the tile in shared memory while
-//   phase A   its slice's contribution to T (64 x NB, tcgen05.mma M = 64, K = 512) goes to TMEM,
+// before a single element of Y = X^T T can be formed, so the unfused kernels read X twice from
+// HBM.  Here a thread-block cluster of C CTAs shares a tile of 128 tokens; CTA c works on its
+// 512-column slice of the tile:
+//   phase A   the slice's contribution to T (128 x NB, tcgen05.mma M = 128, K = 512) goes to TMEM;
+//             X streams through a ring of shared-memory slots (first read, from HBM, marked
+//             evict-last for L2) and every slot is released as soon as its MMAs have read it,
 //   exchange  the C partial sums are added up through distributed shared memory in two one-way
-//             hops (st.async): each row of the tile is summed in rank order by the CTA that owns
-//             it, and the sum is sent to every CTA, so all of them hold the same T,
-//   phase C   Y_slice (512 x NB, kept in TMEM across all tiles of the work item) += X_slice^T T
-//             (tcgen05.mma M = 128, the resident X boxes read as an MN-major operand).
-// X therefore crosses HBM once per power step.  A work item is (layer, token slab); the slab's
-// partial Y leaves TMEM once, at the end of the item, and the slabs are summed by the panel QR.
+//             hops (st.async): groups of eight token rows are summed in rank order by the CTA that
+//             owns them, which writes the bf16 hi/lo parts of the sums straight into the T operand
+//             buffer of every CTA of the cluster,
+//   phase C   Y_slice (512 x NB, kept in TMEM across all tiles of the work item) += X_slice^T T;
+//             the slice is fetched a second time through a second, smaller ring -- a few boxes
+//             behind the first read, so it comes from L2 (measured: a line survives 20 to 50 MB of
+//             streaming traffic, and this lag is about one tile per CTA).
+// An earlier version kept the tile resident in shared memory between the phases; the exchange
+// takes about 2 us, the ring held 2.5 tiles of 64 KiB, and that residency, not the arithmetic,
+// bounded it at 3.6 TB/s.  A work item is (layer, token slab); the slab's partial Y leaves TMEM
+// once, at the end of the item, and the slabs are summed by the panel QR.
 //
 // As in the unfused kernels Q and T are fp32 quantities carried as hi + lo bf16 pairs in NB = 2 NP
 // operand columns (NP = r rounded up to 8), products exact, accumulation fp32.
 //
-// Status: correct (same parity tests as the two-sweep kernels) but not faster, so it is an option
-// ("extract_fused"), off by default.  Measured on B200 at d_in = 4096, r = 16, clusters of 8
-// (timestamps taken inside the kernel): the exchange takes 1.35 us from the last phase-A MMA to
-// the T operand being ready (it took 4.4 us with remote loads and cluster-scope release arrives),
-// but a tile still takes 3.5 us, because its 32 + 16 tcgen05.mma instructions (M = 64 or 128,
-// N = 32, K = 16) cost about 65 to 80 ns each whatever their size -- neither fewer instructions
-// in the issuing thread nor independent accumulators changed that.  64 KiB per 3.5 us is 19 GB/s
-// per CTA, 2.3 TB/s over the 120 CTAs of 15 resident clusters, against the 6.8 TB/s at which the
-// two-sweep kernels read X twice (they need one such instruction per 4 KiB of X and run two CTAs
-// per SM).  A fused step needs a product shape with more work per instruction (the 256-wide N
-// side on X, tiles of 128 or more tokens) before it can win.
-//
-// Roles in a CTA: warp 0 TMA producer (Q slice once per item, X slots of [64 tokens][128 columns]
-// through a ring), warp 1 MMA issuer (phase A of tile i+1 is issued before phase C of tile i so the
-// exchange of one tile overlaps the loads and phase A of the next), two groups of four epilogue warps
-// that take alternate tiles (TMEM -> exchange -> T operand; group 0 also writes Y out).  Every wait is bounded; a wait that runs out sets the status
-// word and the CTA leaves through the common exit (copies drained, cluster barrier, TMEM freed).
+// Roles in a CTA: warp 0 TMA producer of ring A (and of the Q slice, once per item), warp 10 TMA
+// producer of ring C, warp 1 MMA issuer (all lanes run the loop, an elected lane issues; phase A of
+// tile i+1 is issued before phase C of tile i so that the exchange of one tile overlaps the loads
+// and phase A of the next), two groups of four epilogue warps that take alternate tiles (TMEM ->
+// exchange; group 0 also writes Y out).  Every wait is bounded; a wait that runs out sets the
+// status word and the CTA leaves through the common exit (cluster barrier, TMEM freed).
 #include <cuda.h>
 
 #include "agzo_ptx.cuh"
@@ -44,24 +40,30 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kFzThreads = 64 + 2 * 128;   // producer warp, MMA warp, two epilogue groups of four warps
-constexpr int kTT = 64;                    // tokens per tile
+constexpr int kFzThreads = 11 * 32;        // producer A, MMA, two epilogue groups of four warps, producer C
+constexpr int kWarpProdC = 10;
+constexpr int kTT = 128;                   // tokens per tile
+constexpr int kGroups = kTT / 8;           // token groups of a tile (the unit of ownership in the exchange)
 constexpr int kSliceCols = 512;            // columns of X per CTA
 constexpr int kMBlocks = kSliceCols / 128; // M blocks of phase C
-constexpr int kSlotBytes = 16 * 1024;      // [64 tokens][128 columns] as two boxes of 64 columns
-constexpr int kBoxBytes = 8 * 1024;
-constexpr int kMaxRing = 12;
-constexpr int kRsFloats = 1792;            // C * ceil(8 / C) * 8 * NP floats at most (C = 7, NP = 16)
+constexpr int kSlotBytes = 16 * 1024;      // ring A: [128 tokens][64 columns]; ring C: [64 tokens][128 columns]
+constexpr int kBoxBytes = 8 * 1024;        // one TMA box of 64 tokens x 64 columns
+constexpr int kRingA = 5, kRingC = 4;
+constexpr int kMaxRing = 8;
+constexpr int kLook = 2;                   // phase A runs up to this many tiles ahead of phase C
+constexpr int kBuf = kLook + 1;            // T partial (TMEM) and T operand (shared memory) buffers in rotation
+constexpr int kRs = 2;                     // exchange buffers in rotation
+constexpr int kRsFloats = 2688;            // C * ceil(16 / C) * 8 * NP floats at most (C = 7, NP = 16)
+constexpr int kTtBytes = 32 * 256;         // T operand: up to 32 rows of 128 tokens
 constexpr uint32_t kFzTmemCols = 256;
-constexpr int kLook = 1;                   // phase A runs this many tiles ahead of phase C
-constexpr int kBuf = kLook + 1;            // T partial / exchange / T operand buffers in rotation
 
 struct FzShared {
-  uint64_t x_full[kMaxRing], x_empty[kMaxRing];
+  uint64_t xa_full[kMaxRing], xa_empty[kMaxRing];
+  uint64_t xc_full[kMaxRing], xc_empty[kMaxRing];
   uint64_t qb_full, qb_empty;
   uint64_t tp_full[kBuf], tp_empty[kBuf];     // T partial in TMEM
   uint64_t tt_full[kBuf];                     // T operand in shared memory: the owners' sums have landed
-  uint64_t rs_full[kBuf];                     // exchange: the contributions to the rank indices I own have landed
+  uint64_t rs_full[kRs];                      // exchange: the contributions to the token groups I own have landed
   uint64_t y_full, y_free;
   uint32_t tmem_base;
   int failed;
@@ -95,7 +97,7 @@ __device__ __forceinline__ uint32_t swz(int i, int j) {
 }
 
 __global__ void __launch_bounds__(kFzThreads, 1)
-fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, int ring, int pf, DevStatus* status) {
+fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, DevStatus* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ FzShared sh;
@@ -103,22 +105,24 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
   const int rank = (int)cluster_ctarank();
   const int cluster = (int)cluster_id_x(), nclusters = (int)cluster_count_x();
   const int col0 = rank * kSliceCols;
-  // shared-memory carve-up: X ring | Q slice (8 boxes of [NB][64]) | T operand x2 | exchange buffers x2
-  uint8_t* sX = base;
-  uint8_t* sQ = sX + (size_t)ring * kSlotBytes;
+  // shared-memory carve-up: ring A | ring C | Q slice (8 boxes of [NB][64]) | T operand x kBuf | exchange buffers x kRs | staging
+  uint8_t* sXA = base;
+  uint8_t* sXC = sXA + (size_t)kRingA * kSlotBytes;
+  uint8_t* sQ = sXC + (size_t)kRingC * kSlotBytes;
   // NB is a per-layer quantity; the regions are sized for NB = 32
   uint8_t* sTt = sQ + 8 * 32 * 128;
-  float* sRs = reinterpret_cast<float*>(sTt + kBuf * 32 * 128);  // kBuf x [C][cpo][8][NP] floats
-  uint8_t* sStage = reinterpret_cast<uint8_t*>(sRs + kBuf * kRsFloats);   // 512 bytes per epilogue warp
+  float* sRs = reinterpret_cast<float*>(sTt + kBuf * kTtBytes);   // kRs x [C][cpo][8][NP] floats
+  uint8_t* sStage = reinterpret_cast<uint8_t*>(sRs + kRs * kRsFloats);   // 512 bytes per epilogue warp
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < ring; ++s) { mbar_init(&sh.x_full[s], 1); mbar_init(&sh.x_empty[s], 1); }
+    for (int s = 0; s < kRingA; ++s) { mbar_init(&sh.xa_full[s], 1); mbar_init(&sh.xa_empty[s], 1); }
+    for (int s = 0; s < kRingC; ++s) { mbar_init(&sh.xc_full[s], 1); mbar_init(&sh.xc_empty[s], 1); }
     mbar_init(&sh.qb_full, 1); mbar_init(&sh.qb_empty, 1);
     for (int p = 0; p < kBuf; ++p) {
       mbar_init(&sh.tp_full[p], 1); mbar_init(&sh.tp_empty[p], 4);
       mbar_init(&sh.tt_full[p], 1);
-      mbar_init(&sh.rs_full[p], 1);
     }
+    for (int p = 0; p < kRs; ++p) mbar_init(&sh.rs_full[p], 1);
     mbar_init(&sh.y_full, 1); mbar_init(&sh.y_free, 4);
     sh.failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -133,7 +137,8 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
 
   if (warp == 0) {
     if (lane == 0) {
-      // ------------------------------------------------ TMA producer
+      // ------------------------------------------------ TMA producer, ring A: the first read of X (and the Q slice)
+      const uint64_t keep = l2_policy_evict_last();
       int ns = 0, ic = 0;
       bool ok = true;
       FzItem it;
@@ -146,30 +151,57 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         tmap_acquire(map_q);
         const int live = min(kSliceCols, L.d_in - col0);
         const int nq = (live + 63) / 64;                 // live 64-column boxes of this slice
-        const int mb = (live + 127) / 128;               // live M blocks
         const int q_box = L.NB * 128;
         if (ic > 0 && !mbar_wait(&sh.qb_empty, (ic - 1) & 1)) { ok = false; break; }
         mbar_expect_tx(&sh.qb_full, (uint32_t)(nq * q_box));
         for (int j = 0; j < nq; ++j) tma_load_2d(sQ + (size_t)j * q_box, map_q, col0 + 64 * j, 0, &sh.qb_full);
         for (int tile = 0; tile < it.ntiles && ok; ++tile) {
           const int t0 = it.t_begin + tile * kTT;
-          for (int b = 0; b < mb; ++b, ++ns) {
-            const int s = ns % ring, u = ns / ring;
-            if (u > 0 && !mbar_wait(&sh.x_empty[s], (u - 1) & 1)) { ok = false; break; }
-            uint8_t* slot = sX + (size_t)s * kSlotBytes;
-            mbar_expect_tx(&sh.x_full[s], kSlotBytes);
-            tma_load_2d(slot, map_x, col0 + 128 * b, t0, &sh.x_full[s]);
-            tma_load_2d(slot + kBoxBytes, map_x, col0 + 128 * b + 64, t0, &sh.x_full[s]);
-            if (tile + pf < it.ntiles) {     // the tile `pf` steps ahead starts its way from DRAM to L2 now
-              tma_prefetch_2d(map_x, col0 + 128 * b, t0 + pf * kTT);
-              tma_prefetch_2d(map_x, col0 + 128 * b + 64, t0 + pf * kTT);
-            }
+          for (int j = 0; j < nq; ++j, ++ns) {
+            const int s = ns % kRingA, u = ns / kRingA;
+            if (u > 0 && !mbar_wait(&sh.xa_empty[s], (u - 1) & 1)) { ok = false; break; }
+            uint8_t* slot = sXA + (size_t)s * kSlotBytes;
+            mbar_expect_tx(&sh.xa_full[s], kSlotBytes);
+            tma_load_2d_hint(slot, map_x, col0 + 64 * j, t0, &sh.xa_full[s], keep);
+            tma_load_2d_hint(slot + kBoxBytes, map_x, col0 + 64 * j, t0 + 64, &sh.xa_full[s], keep);
           }
         }
       }
       if (!ok) sh.failed = 1;
       if (!ok || sh.failed) {   // leaving early: the copies in flight must land before the CTA goes away
-        for (int k = ns > ring ? ns - ring : 0; k < ns; ++k) mbar_wait(&sh.x_full[k % ring], (k / ring) & 1);
+        for (int k = ns > kRingA ? ns - kRingA : 0; k < ns; ++k) mbar_wait(&sh.xa_full[k % kRingA], (k / kRingA) & 1);
+      }
+    }
+  } else if (warp == kWarpProdC) {
+    if (lane == 0) {
+      // ------------------------------------------------ TMA producer, ring C: the second read, a few boxes behind, from L2
+      const uint64_t drop = l2_policy_evict_first();
+      int ns = 0;
+      bool ok = true;
+      FzItem it;
+      for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters) {
+        const DevLayer& L = *it.L;
+        const void* map_x = L.tmaps;
+        tmap_acquire(map_x);
+        const int live = min(kSliceCols, L.d_in - col0);
+        const int mb = (live + 127) / 128;               // live M blocks
+        for (int tile = 0; tile < it.ntiles && ok; ++tile) {
+          const int t0 = it.t_begin + tile * kTT;
+          for (int b = 0; b < mb && ok; ++b) {
+            for (int h = 0; h < 2; ++h, ++ns) {
+              const int s = ns % kRingC, u = ns / kRingC;
+              if (u > 0 && !mbar_wait(&sh.xc_empty[s], (u - 1) & 1)) { ok = false; break; }
+              uint8_t* slot = sXC + (size_t)s * kSlotBytes;
+              mbar_expect_tx(&sh.xc_full[s], kSlotBytes);
+              tma_load_2d_hint(slot, map_x, col0 + 128 * b, t0 + 64 * h, &sh.xc_full[s], drop);
+              tma_load_2d_hint(slot + kBoxBytes, map_x, col0 + 128 * b + 64, t0 + 64 * h, &sh.xc_full[s], drop);
+            }
+          }
+        }
+      }
+      if (!ok) sh.failed = 1;
+      if (!ok || sh.failed) {
+        for (int k = ns > kRingC ? ns - kRingC : 0; k < ns; ++k) mbar_wait(&sh.xc_full[k % kRingC], (k / kRingC) & 1);
       }
     }
   } else if (warp == 1) {
@@ -183,67 +215,91 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       int ic = 0;
       bool ok = true;
       FzItem it;
-      const uint32_t sq_addr = smem_u32(sQ), sx_addr = smem_u32(sX), stt_addr = smem_u32(sTt);
+      const uint32_t sq_addr = smem_u32(sQ), sxa_addr = smem_u32(sXA), sxc_addr = smem_u32(sXC), stt_addr = smem_u32(sTt);
       for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters, ++ic) {
         const DevLayer& L = *it.L;
         const int NB = L.NB;
         const int live = min(kSliceCols, L.d_in - col0);
-        const int mb = (live + 127) / 128;
+        const int nq = (live + 63) / 64, mb = (live + 127) / 128;
         const uint32_t q_box = (uint32_t)NB * 128u;
-        const uint32_t idesc_a = instr_desc(64, NB, 0, 0);
-        const uint32_t idesc_c = instr_desc(128, NB, 1, 0);      // A = resident X boxes read as X^T
+        const uint32_t idesc_a = instr_desc(128, NB, 0, 0);
+        const uint32_t idesc_c = instr_desc(128, NB, 1, 0);      // A = X boxes read as X^T
         const uint32_t tp_col = (uint32_t)(kMBlocks * NB);       // T partials sit after the Y accumulators
         if (!mbar_wait_warp(&sh.qb_full, ic & 1)) { ok = false; break; }
         if (ic > 0 && !mbar_wait_warp(&sh.y_free, (ic - 1) & 1)) { ok = false; break; }
-        for (int step = 0; step < it.ntiles + kLook && ok; ++step) {
-          if (step < it.ntiles) {
-            // phase A of tile `step`
+        // The two phases are issued as their operands arrive, whichever is ready: phase A of tile a_tile box by
+        // box from ring A, phase C of tile c_tile half a block at a time from ring C.  Two rules order them:
+        // phase C of a tile needs its T operand (tt_full), and phase A may run at most kLook tiles ahead of
+        // phase C -- the T partial and T operand buffers rotate over kBuf = kLook + 1 tiles, and phase A of tile
+        // i + kBuf, being issued after phase C of tile i, completes after the last read of the buffers of tile i.
+        // The exchange buffers rotate over kRs = 2 tiles only: phase A of tile i + 2 waits until the sums of
+        // tile i have landed here (tt_full seen), i.e. until every owner is done with its exchange buffer.
+        int a_tile = 0, a_box = 0, c_tile = 0, c_unit = 0;
+        bool tt_ready = false;
+        uint32_t acc_a = 0u;
+        int idle = 0;
+        unsigned long long idle_t0 = 0;
+        while (c_tile < it.ntiles) {
+          bool did = false;
+          if (a_tile < it.ntiles && (a_tile <= c_tile + 1 || (a_tile == c_tile + 2 && tt_ready))) {
             const int p = ta % kBuf, u2 = ta / kBuf;
-            if (u2 > 0 && !mbar_wait_warp(&sh.tp_empty[p], (u2 - 1) & 1)) { ok = false; break; }
-            const uint32_t d_tp = tmem + tp_col + (uint32_t)(p * NB);
-            uint32_t acc = 0u;
-            for (int b = 0; b < mb && ok; ++b, ++na) {
-              const int s = na % ring, u = na / ring;
-              if (!mbar_wait_warp(&sh.x_full[s], u & 1)) { ok = false; break; }
+            if (a_box == 0 && u2 > 0 && !mbar_wait_warp(&sh.tp_empty[p], (u2 - 1) & 1)) { ok = false; break; }
+            const int s = na % kRingA, u = na / kRingA;
+            if (mbar_test_warp(&sh.xa_full[s], u & 1)) {
               tc_fence_after();
-              const uint32_t slot = sx_addr + (uint32_t)s * kSlotBytes;
-              for (int half = 0; half < 2; ++half) {
-                if (128 * b + 64 * half >= live) break;          // box beyond d_in: its Q box was never loaded
-                const uint64_t xd = smem_desc(slot + half * kBoxBytes, 0, 1024);
-                const uint64_t qd = smem_desc(sq_addr + (uint32_t)(2 * b + half) * q_box, 0, 1024);
+              const uint32_t d_tp = tmem + tp_col + (uint32_t)(p * NB);
+              const uint64_t xd = smem_desc(sxa_addr + (uint32_t)s * kSlotBytes, 0, 1024);
+              const uint64_t qd = smem_desc(sq_addr + (uint32_t)a_box * q_box, 0, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {                 // 16 columns = 32 bytes = 2 descriptor units further
-                  mma_bf16_if(go, d_tp, xd + (uint64_t)(2 * kk), qd + (uint64_t)(2 * kk), idesc_a, acc);
-                  acc = 1u;
-                }
+              for (int kk = 0; kk < 4; ++kk) {                 // 16 columns = 32 bytes = 2 descriptor units further
+                mma_bf16_if(go, d_tp, xd + (uint64_t)(2 * kk), qd + (uint64_t)(2 * kk), idesc_a, acc_a);
+                acc_a = 1u;
               }
+              mma_commit_if(go, &sh.xa_empty[s]);              // the slot is free once these MMAs have read it
+              ++na;
+              if (++a_box == nq) {
+                mma_commit_if(go, &sh.tp_full[p]);
+                if (a_tile == it.ntiles - 1) mma_commit_if(go, &sh.qb_empty);   // last use of this item's Q slice
+                a_box = 0; acc_a = 0u; ++a_tile; ++ta;
+              }
+              did = true;
             }
-            if (!ok) break;
-            mma_commit_if(go, &sh.tp_full[p]);
-            if (step == it.ntiles - 1) mma_commit_if(go, &sh.qb_empty);   // last use of this item's Q slice
-            ++ta;
           }
-          if (step >= kLook) {
-            // phase C of tile `step - kLook`
+          if (c_tile < a_tile) {
             const int p = tcn % kBuf, u2 = tcn / kBuf;
-            if (!mbar_wait_cluster_warp(&sh.tt_full[p], u2 & 1)) { ok = false; break; }
-            fence_proxy_async();      // the operand was written by generic-proxy stores of the owners
-            tc_fence_after();
-            const uint64_t td = smem_desc(stt_addr + (uint32_t)p * 32u * 128u, 0, 1024);
-            for (int b = 0; b < mb; ++b, ++nc) {
-              const int s = nc % ring;
-              // 16 tokens = two 8-row swizzle atoms = 2048 bytes = 128 descriptor units further down both boxes
-              const uint64_t xd = smem_desc(sx_addr + (uint32_t)s * kSlotBytes, kBoxBytes, 1024);
+            if (!tt_ready && mbar_test_cluster_warp(&sh.tt_full[p], u2 & 1)) {
+              fence_proxy_async();      // the operand was written by the owners' stores, not by the async proxy
+              tt_ready = true;
+            }
+            const int s = nc % kRingC, u = nc / kRingC;
+            if (tt_ready && mbar_test_warp(&sh.xc_full[s], u & 1)) {
+              tc_fence_after();
+              const int b = c_unit >> 1, h = c_unit & 1;
               const uint32_t d_y = tmem + (uint32_t)(b * NB);
+              // 16 tokens = two 8-row swizzle atoms = 2048 bytes = 128 descriptor units further down both boxes;
+              // the T operand holds 64 tokens per 128-byte atom column, NB rows each
+              const uint64_t xd = smem_desc(sxc_addr + (uint32_t)s * kSlotBytes, kBoxBytes, 1024);
+              const uint64_t th = smem_desc(stt_addr + (uint32_t)p * kTtBytes + (uint32_t)(h * NB * 128), 0, 1024);
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk)
-                mma_bf16_if(go, d_y, xd + (uint64_t)(128 * kk), td + (uint64_t)(2 * kk), idesc_c,
-                            (step > kLook || kk > 0) ? 1u : 0u);
-              mma_commit_if(go, &sh.x_empty[s]);
+                mma_bf16_if(go, d_y, xd + (uint64_t)(128 * kk), th + (uint64_t)(2 * kk), idesc_c,
+                            (c_tile > 0 || h > 0 || kk > 0) ? 1u : 0u);
+              mma_commit_if(go, &sh.xc_empty[s]);
+              ++nc;
+              if (++c_unit == 2 * mb) { c_unit = 0; ++c_tile; ++tcn; tt_ready = false; }
+              did = true;
             }
-            ++tcn;
+          }
+          if (did) {
+            idle = 0;
+          } else if (++idle >= 1024) {       // nothing was ready a thousand times over: look at the clock
+            const unsigned long long now = global_ns();
+            if (idle == 1024) idle_t0 = now;
+            if (now - idle_t0 > kWaitCapNs) { ok = false; break; }
+            idle = 1025;
           }
         }
+        if (!ok) break;
         if (ok) mma_commit_if(go, &sh.y_full);
       }
       if (!ok) sh.failed = 1;
@@ -265,15 +321,16 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       const int live = min(kSliceCols, L.d_in - col0);
       const int mb = (live + 127) / 128;
       const uint32_t tp_col = (uint32_t)(kMBlocks * NB);
-      const int cpo = (kTT / 8 + C - 1) / C;   // token groups of a tile per owner, at most
+      const int cpo = (kGroups + C - 1) / C;   // token groups of a tile per owner, at most
       for (int tile = 0; tile < it.ntiles && ok; ++tile, ++te) {
-        const int p = te % kBuf, u2 = te / kBuf;
+        const int p = te % kBuf, u2 = te / kBuf;     // T partial and T operand buffers
+        const int pr = te % kRs, ur = te / kRs;      // exchange buffer
         if ((te & 1) != grp) continue;
         ok = mbar_wait(&sh.tp_full[p], u2 & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        // an M = 64 accumulator keeps row 16q + i in lane 32q + i for i < 16; lanes 16..31 of a warp hold nothing.
+        // an M = 128 accumulator keeps row R in TMEM lane R: this thread holds token row 32q + lane of the tile.
         // The buffer's NB columns are [hi parts | lo parts]: one load of up to 32 columns brings both.
         float tsum[16];
         {
@@ -299,39 +356,42 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         //                   lo parts and writes them straight into the T operand of every CTA of the cluster:
         //                   eight tokens of one operand row are one 16-byte piece.  The bytes are counted on
         //                   the receiver's tt_full barrier, which is what its MMA warp waits for.
-        // No buffer needs a "free" signal.  A peer sends tile i + kBuf's data only after its phase A of that
-        // tile has completed, hence (its MMAs run in order) after its phase C of tile i, hence after it has
-        // received my tile-i sums, which I sent after reading the tile-i contributions.  And the T operand
-        // buffer of a receiver is free once its phase A of tile i is complete (phase C of tile i - kBuf was
-        // issued before it), which is before it sends the contribution that my sum of tile i waits for.
-        float* rs = sRs + p * kRsFloats;          // [C sources][cpo groups][8 tokens][NP]
-        const int my_c = (kTT / 8 - rank + C - 1) / C;      // token groups of a tile that this CTA owns
+        // No buffer needs a "free" signal.  A peer sends the contributions of tile i + 2 only after its phase A
+        // of that tile has completed, which it issued after it had received the tile-i sums of every owner, mine
+        // among them, and I send those after reading the tile-i contributions.  And the T operand buffer of a
+        // receiver is free for tile i + kBuf once its phase A of that tile is complete (its phase C of tile i was
+        // issued before it and the MMAs run in order), which is before it sends the contribution that the
+        // owners' sums of tile i + kBuf wait for.
+        float* rs = sRs + pr * kRsFloats;         // [C sources][cpo groups][8 tokens][NP]
+        const int my_c = (kGroups - rank + C - 1) / C;      // token groups of a tile that this CTA owns
         if (et == 0) {
-          mbar_expect_tx(&sh.rs_full[p], (uint32_t)(C * my_c * 8 * NP * 4));
+          mbar_expect_tx(&sh.rs_full[pr], (uint32_t)(C * my_c * 8 * NP * 4));
           mbar_expect_tx(&sh.tt_full[p], (uint32_t)(NP * kTT * 4));
         }
-        if (lane < 16) {
-          const int R = 16 * q + lane, j = R >> 3, dest = j % C, jc = j / C;
+        {
+          const int R = 32 * q + lane, j = R >> 3, dest = j % C, jc = j / C;
           const uint32_t dst = mapa_shared(smem_u32(rs + ((rank * cpo + jc) * 8 + (R & 7)) * NP), (uint32_t)dest);
-          const uint32_t bar = mapa_shared(smem_u32(&sh.rs_full[p]), (uint32_t)dest);
+          const uint32_t bar = mapa_shared(smem_u32(&sh.rs_full[pr]), (uint32_t)dest);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
             if (k4 * 4 < NP)
               st_async_f4(dst + k4 * 16, make_float4(tsum[k4 * 4], tsum[k4 * 4 + 1], tsum[k4 * 4 + 2], tsum[k4 * 4 + 3]),
                           bar);
         }
-        ok = mbar_wait_cluster(&sh.rs_full[p], u2 & 1);
+        ok = mbar_wait_cluster(&sh.rs_full[pr], ur & 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        // Every warp of the group adds the C contributions of an owned token group (lane = (token of the
-        // group, four rank indices); the four warps do the same additions, which is cheaper than handing
-        // the sums over), passes the bf16 parts through its 512-byte staging block so that a lane then
-        // holds one 16-byte piece (eight tokens of one operand row), and sends it to the CTAs d = q mod 4.
+        // The group's four warps share the owned token groups and the destinations: with fewer than four
+        // owned groups two or four warps take the same group (each adds it up again, which is cheaper than
+        // handing the sums over) and send to different CTAs.  Lane = (token of the group, four rank indices)
+        // adds the C contributions, the bf16 parts pass through the warp's 512-byte staging block so that a
+        // lane then holds one 16-byte piece (eight tokens of one operand row), and sends it.
         {
           __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(sStage) + ((grp * 4 + q) * 32 * 8);
-          const uint32_t tt_base = smem_u32(sTt) + (uint32_t)p * 32u * 128u;
+          const uint32_t tt_base = smem_u32(sTt) + (uint32_t)p * kTtBytes;
           const uint32_t tt_bar = smem_u32(&sh.tt_full[p]);
-          for (int jc = 0; jc < my_c; ++jc) {
+          const int nsplit = my_c >= 4 ? 1 : (my_c >= 2 ? 2 : 4);   // warps per owned group
+          for (int jc = q / nsplit; jc < my_c; jc += 4 / nsplit) {
             const int x = lane & 7, kq = lane >> 3;
             if (4 * kq < NP) {
               float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -348,11 +408,13 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
               }
             }
             __syncwarp();
-            if (lane < 2 * NP) {      // operand rows: hi parts 0..NP-1, then lo parts
+            if (lane < 2 * NP) {      // operand rows: hi parts 0..NP-1, then lo parts; 64 tokens per 128-byte atom
               const uint4 piece = *reinterpret_cast<const uint4*>(stage + lane * 8);
               const uint32_t pv[4] = {piece.x, piece.y, piece.z, piece.w};
-              const uint32_t off = tt_base + swz(lane, rank + C * jc);
-              for (int d = q; d < C; d += 4) st_async_u4(mapa_shared(off, (uint32_t)d), pv, mapa_shared(tt_bar, (uint32_t)d));
+              const int j = rank + C * jc;                  // the token group inside the tile
+              const uint32_t off = tt_base + (uint32_t)((j >> 3) * (2 * NP * 128)) + swz(lane, j & 7);
+              for (int d = q % nsplit; d < C; d += nsplit)
+                st_async_u4(mapa_shared(off, (uint32_t)d), pv, mapa_shared(tt_bar, (uint32_t)d));
             }
             __syncwarp();
           }
@@ -394,10 +456,9 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
 
 int g_max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // per cluster size, filled on first use
 
-size_t fz_smem_bytes(int ring) {
-  return (size_t)ring * kSlotBytes + 8 * 32 * 128 + kBuf * 32 * 128 + kBuf * kRsFloats * 4 + 8 * 512 + 1024;
+size_t fz_smem_bytes() {
+  return (size_t)(kRingA + kRingC) * kSlotBytes + 8 * 32 * 128 + kBuf * kTtBytes + kRs * kRsFloats * 4 + 8 * 512 + 1024;
 }
-constexpr int kFzRing = 10;    // as many slots as fit beside the other regions in 227 KiB
 
 }  // namespace
 
@@ -409,7 +470,7 @@ int fused_cluster_size(const agzo_layer& a) { return (a.d_in + kSliceCols - 1) /
 
 cudaError_t fused_init() {
   cudaError_t e = cudaFuncSetAttribute(fused_power_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)fz_smem_bytes(kFzRing));
+                                       (int)fz_smem_bytes());
   return e;
 }
 
@@ -420,7 +481,7 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   for (int i = w.l0; i < w.l1; ++i)
     if (h_dev[i].fz_C == C) items += h_dev[i].slabs;
   if (items == 0) return cudaSuccess;
-  const size_t smem = fz_smem_bytes(kFzRing);
+  const size_t smem = fz_smem_bytes();
   cudaLaunchConfig_t cfg{};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -444,9 +505,8 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   const int nclusters = items < g_max_clusters[C] ? items : g_max_clusters[C];
   cfg.gridDim = dim3((unsigned)(nclusters * C));
   const DevLayer* layers = w.d_layers;
-  int l0 = w.l0, l1 = w.l1, ring = kFzRing;
-  int pf = 2;      // tiles ahead of the loads at which L2 is asked to fetch (no measurable effect between 0 and 4)
-  void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&ring, (void*)&pf, (void*)&d_status};
+  int l0 = w.l0, l1 = w.l1;
+  void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&d_status};
   return cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel, args);
 }
 
