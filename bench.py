@@ -265,7 +265,7 @@ def whole_job_units(per_rank_units: float, world: int) -> float:
 
 
 # ----------------------------------------------------------------------------- sweep
-def sweep_entry(B, cfg, r, Ws, Xs, dev, local, peak, steps=3, wave_bytes=None, label=None):
+def sweep_entry(B, cfg, r, Ws, Xs, dev, local, peak, steps=3, wave_bytes=None, label=None, fused=-1):
     """One short run of the whole step on a resident layer set at rank r: step, extraction and one
     pass (CUDA events), the pass's bandwidth, the device status."""
     Vs = [torch.zeros(r, X.shape[1], dtype=torch.float32, device=dev) for X in Xs]
@@ -274,6 +274,9 @@ def sweep_entry(B, cfg, r, Ws, Xs, dev, local, peak, steps=3, wave_bytes=None, l
     ctx = B.agzo_create(layers, local)
     if wave_bytes is not None:
         B.agzo_set_option(ctx, "wave_bytes", wave_bytes)
+    if fused >= 0:
+        B.agzo_set_option(ctx, "extract_fused", fused)
+    n_fused = sum(1 for c in B.agzo_query_fused(ctx, layers, arr=arr) if c)
     losses = torch.tensor([1.0, 0.999], dtype=torch.float64, device=dev)
     ghat = torch.zeros(1, device=dev)
     stream = torch.cuda.current_stream()
@@ -306,6 +309,7 @@ def sweep_entry(B, cfg, r, Ws, Xs, dev, local, peak, steps=3, wave_bytes=None, l
     return {"workload": label or cfg.name, "r": r, "step_ms": ms_step, "extract_ms": ms_extract, "pass_ms": ms_pass,
             "pass_GBps": gbps, "pass_frac_of_measured_hbm": gbps / peak, "pass_frac_of_nominal_8TBps": gbps / 8000.0,
             "extract_GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6,
+            "layers_with_fused_power_steps": n_fused,
             "device_status": B.status_string(status)}
 
 
@@ -317,15 +321,15 @@ def run_sweep(B, args, cfg_head, Ws, Xs, dev, local, peak):
     out = []
     for r in (1, 4, 64):
         if r != args.rank:
-            out.append(sweep_entry(B, cfg_head, r, Ws, Xs, dev, local, peak))
+            out.append(sweep_entry(B, cfg_head, r, Ws, Xs, dev, local, peak, fused=args.extract_fused))
     Ws.clear(); Xs.clear()
     torch.cuda.empty_cache()
     for cfg, ranks in ((WL.QWEN3_1P7B, (4, 8, 16)), (WL.QWEN3_0P6B, (8,))):
         W2, X2, _, _ = build_layer_set(cfg, 1, dev)
         for r in ranks:
-            out.append(sweep_entry(B, cfg, r, W2, X2, dev, local, peak))
+            out.append(sweep_entry(B, cfg, r, W2, X2, dev, local, peak, fused=args.extract_fused))
         if cfg is WL.QWEN3_0P6B:
-            e = sweep_entry(B, cfg, 8, W2, X2, dev, local, peak, wave_bytes=56 << 20,
+            e = sweep_entry(B, cfg, 8, W2, X2, dev, local, peak, wave_bytes=56 << 20, fused=args.extract_fused,
                             label=cfg.name + ", extraction in waves of at most 56 MB of activations (X stays in L2 "
                                              "across the sweeps of a wave)")
             out.append(e)
@@ -346,7 +350,8 @@ def main():
     ap.add_argument("--extract-path", type=int, default=0)
     ap.add_argument("--wave-mb", type=int, default=-1)
     ap.add_argument("--extract-streams", type=int, default=2)
-    ap.add_argument("--extract-fused", type=int, default=0)
+    ap.add_argument("--extract-fused", type=int, default=-1,
+                    help="-1: the library's default (fused power steps where a layer allows); 0/1/2: the option")
     ap.add_argument("--alias-inputs", action="store_true",
                     help="q/k/v and gate/up of a block read one activation buffer each (as in a real block)")
     ap.add_argument("--share-inputs", type=int, default=1)
@@ -412,7 +417,8 @@ def main():
     B.agzo_set_option(ctx, "extract_path", args.extract_path)
     B.agzo_set_option(ctx, "rmw_path", args.rmw_path)
     B.agzo_set_option(ctx, "extract_streams", args.extract_streams)
-    B.agzo_set_option(ctx, "extract_fused", args.extract_fused)
+    if args.extract_fused >= 0:
+        B.agzo_set_option(ctx, "extract_fused", args.extract_fused)
     B.agzo_set_option(ctx, "share_inputs", args.share_inputs)
     B.agzo_set_option(ctx, "rmw_tc_slots", args.rmw_slots)
     B.agzo_set_option(ctx, "rmw_tc_inflight", args.rmw_inflight)
@@ -470,7 +476,12 @@ def main():
     if st_warm != B.AGZO_OK:
         raise SystemExit("device status after warm-up: " + B.status_string(st_warm))
     tc_used = args.extract_path != 1
-    dom_class = B.KC_TC_XT_T if tc_used else B.KC_XT_T
+    # which layers run their power steps in the fused kernel (the library decides by shape and device);
+    # the kernel class that moves most of the step's bytes is the one timed launch by launch
+    fz = B.agzo_query_fused(ctx, layers, arr=arr) if args.method == "agzo" else [0] * len(layers)
+    x_fused = sum({X.data_ptr(): X.numel() * X.element_size() for X, c in zip(Xs, fz) if c}.values())
+    fused_dominant = tc_used and K_POWER * x_fused > work["x_bytes"] * (K_POWER + 1) - K_POWER * x_fused
+    dom_class = B.KC_FUSED_POWER if fused_dominant else (B.KC_TC_XT_T if tc_used else B.KC_XT_T)
     B.agzo_read_counters(ctx)
     sampler = ClockSampler(local) if rank == 0 else None
     ms_step = timed(step, args.steps, 100)
@@ -529,7 +540,15 @@ def main():
 
     status = B.agzo_poll(ctx)
     peak, peak_kind = measured_peaks()
-    x_bytes_per_launch = work["x_bytes"] * (K_POWER + 1) / max(dom_n / max(args.steps, 1), 1)
+    if fused_dominant:     # K passes over the fused layers' X per step
+        dom_bytes_per_step = K_POWER * x_fused
+        dom_kernel = "fused_power_step_kernel"
+        dom_name = dom_kernel + " (Y = X^T (X Q), X crossing HBM once)"
+    else:                  # the sweep Y = X^T T: once over every X, K times more over the unfused layers' X
+        dom_bytes_per_step = work["x_bytes"] + K_POWER * (work["x_bytes"] - x_fused)
+        dom_kernel = "tc_xt_t_kernel" if tc_used else "xt_t_kernel"
+        dom_name = dom_kernel + " (Y = X^T T)"
+    x_bytes_per_launch = dom_bytes_per_step / max(dom_n / max(args.steps, 1), 1)
     dom_avg_ms = dom_ms / max(dom_n, 1)
     achieved = x_bytes_per_launch / (dom_avg_ms * 1e-3) / 1e9 if dom_n else None
 
@@ -553,15 +572,17 @@ def main():
                     "frac_of_%s_hbm" % peak_kind: work["rmw_bytes_per_pass"] / ms_perturb / 1e6 / peak,
                     "frac_of_nominal_8TBps": work["rmw_bytes_per_pass"] / ms_perturb / 1e6 / 8000.0},
             "extract": {"TFLOPs_algorithmic": work["extract_flops"] / ms_extract / 1e9,
-                        "GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6},
-            "roofline": {"kernel": ("tc_xt_t_kernel" if tc_used else "xt_t_kernel") + " (Y = X^T T)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                        "GBps_fused_bytes": work["extract_bytes_fused"] / ms_extract / 1e6,
+                        "layers_with_fused_power_steps": sum(1 for c in fz if c),
+                        "cluster_sizes": sorted(set(c for c in fz if c))},
+            "roofline": {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                          "frac_of_nominal_8TBps": (achieved / 8000.0) if achieved else None,
                          "peak_kind": peak_kind,
                          "peak_note": "the peak is the copy rate measured on this pool (a read-and-write stream): a "
                                       "reference rate, not a ceiling -- a read-only sweep can exceed it",
-                         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE["tc_xt_t_kernel"] * x_bytes_per_launch
-                                     if tc_used and dom_n else None),
+                         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE[dom_kernel] * x_bytes_per_launch
+                                     if dom_kernel in TRAFFIC_PER_ALGORITHMIC_BYTE and dom_n else None),
                          "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the "
                                          "first 4 blocks of this workload, scaled by the X bytes a launch reads",
                          "launches": dom_n, "avg_ms": dom_avg_ms,

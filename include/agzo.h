@@ -141,8 +141,13 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * "share_inputs" 1 (default) = consecutive layers whose X is the same buffer (same pointer, pitch,
  * m, d_in: q/k/v or gate/up of a transformer block) are served by one sweep over X per product,
  * with identical results; 0 = every layer sweeps its X itself;
- * "extract_fused" 1 = layers with r <= 16 and d_in <= 4096 on the tensor-core path run each
- * power step in the fused kernel that reads X once (thread-block clusters); 0 = off;
+ * "extract_fused" 1 = layers with r <= 16 and d_in <= 12288 on the tensor-core path run each
+ * power step in the fused kernel in which X crosses HBM once (thread-block clusters of
+ * ceil(d_in / 512) CTAs, or ceil(d_in / 768)), where that cluster size keeps at least 70 % of
+ * the device's SMs busy; 2 = the same without the last condition (every cluster size
+ * the device can launch) and also for layers that share their X with a neighbour (with 1 those
+ * stay with the sweeps that serve the whole group); 0 = off: two sweeps over X per power step.
+ * Default 1;
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
  * "extract_streams" 2 (default) = alternate waves use two scratch regions and two helper
  * streams forked from and joined to the caller's stream, so that one wave's short kernels
@@ -198,6 +203,21 @@ typedef enum agzo_kernel_class {
  * are reset.  Any output pointer may be NULL.  Synchronises with the timed events only.   */
 agzo_status agzo_read_counters(agzo_ctx* ctx, double* h_ms, int64_t* h_timed_launches,
                                int64_t* h_total_launches);
+
+/* Inspection aid.  Plans the layer array as agzo_extract_subspace would (the plan is kept for
+ * the next call with the same array; its tables are uploaded on `stream`) and writes, per layer,
+ * the thread-block cluster size with which its power steps run in the fused kernel, 0 for a
+ * layer served by the two-sweep kernels (no X, the "extract_fused" / "extract_path" options,
+ * its shape, or an X shared with a neighbouring layer).  h_cluster: host, n entries.  Launches
+ * no kernel.                                                                               */
+agzo_status agzo_query_fused(agzo_ctx* ctx, const agzo_layer* h_layers, int n, int32_t* h_cluster,
+                             void* stream);
+
+/* Inspection aid.  h_clusters[C], C = 1..16 (17 host entries, entry 0 is 0): how many thread-block
+ * clusters of C CTAs of the fused power-step kernel the context's device holds at once (a cluster
+ * lives inside one GPC, so the answer depends on the chip's GPC sizes); all 0 where the tensor-core
+ * path is unavailable.  This is what "extract_fused" = 1 weighs when it picks a layer's cluster size. */
+agzo_status agzo_query_cluster_capacity(agzo_ctx* ctx, int32_t* h_clusters);
 
 /* Waits for the stream work of this context issued so far on `stream` and returns the
  * device status word: AGZO_OK, AGZO_WARN_RANK_DEFICIENT or AGZO_ERR_TIMEOUT; the word is

@@ -32,7 +32,7 @@ EXPORTS = [
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
     "agzo_extract_subspace_static", "agzo_fill_gaussian_basis", "agzo_set_allreduce",
-    "agzo_debug_wait_timeout",
+    "agzo_debug_wait_timeout", "agzo_query_fused", "agzo_query_cluster_capacity",
 ]
 KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC, KC_FUSED_POWER = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
@@ -101,6 +101,8 @@ def lib() -> C.CDLL:
         "agzo_read_counters": (i32, [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)]),
         "agzo_set_allreduce": (i32, [vp, ALLREDUCE_FN, vp, i64]),
         "agzo_debug_wait_timeout": (i32, [vp, vp]),
+        "agzo_query_fused": (i32, [vp, LP, i32, C.POINTER(C.c_int32), vp]),
+        "agzo_query_cluster_capacity": (i32, [vp, C.POINTER(C.c_int32)]),
         "agzo_extract_subspace_static": (i32, [vp, i64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                C.c_int32, u64, u32, vp, i64, vp, vp]),
     }
@@ -221,6 +223,21 @@ def agzo_read_counters(ctx: Context):
     _check(lib().agzo_read_counters(ctx.handle, C.byref(ms), C.byref(nt), C.byref(na)),
            "agzo_read_counters")
     return ms.value, nt.value, na.value
+
+
+def agzo_query_fused(ctx: Context, layers, stream=None, arr=None):
+    """Per layer: the cluster size of the fused power-step kernel, 0 = two-sweep kernels."""
+    arr = arr if arr is not None else layer_array(layers)
+    out = (C.c_int32 * len(layers))()
+    _check(lib().agzo_query_fused(ctx.handle, arr, len(layers), out, _stream_ptr(stream)), "agzo_query_fused")
+    return list(out)
+
+
+def agzo_query_cluster_capacity(ctx: Context):
+    """[0, clusters of 1 CTA, of 2 CTAs, ..., of 16 CTAs] of the fused kernel resident at once."""
+    out = (C.c_int32 * 17)()
+    _check(lib().agzo_query_cluster_capacity(ctx.handle, out), "agzo_query_cluster_capacity")
+    return list(out)
 
 
 def agzo_poll(ctx: Context, stream=None) -> int:

@@ -54,7 +54,8 @@ struct PlanOpts {
   int rmw_tc_panels;     // column panels per work item of the tensor-core pass (1 or 2)
   int rmw_stage_r;       // 0: stage R in scratch when some rank exceeds 16; 1: never; 2: always
   bool tc_available;
-  bool extract_fused;    // power steps of eligible layers run in the fused single-pass kernel
+  int extract_fused;     // 1: power steps of eligible layers run in the fused single-pass kernel; 2: also on
+                         // cluster sizes that leave much of the device idle
   bool share_inputs;     // consecutive layers with the same X are served by one sweep
   int extract_regions;   // 1: waves run one after another; 2: alternate waves use two scratch regions
                          // and two helper streams, so one wave's small kernels overlap the other's sweeps
@@ -204,10 +205,13 @@ void slab_shape(const agzo_layer& a, bool tc, bool long_slabs, int* slabs, int* 
 }
 
 // scratch bytes one layer needs for extraction (0 when it has no X)
-size_t layer_scratch(const agzo_layer& a, bool tc, bool long_slabs, bool with_panels = true) {
+// y_parts_min: room for at least that many partial sums of Y (the fused power step leaves one per share of
+// its launch that meets the layer, which can be more than the slabs of X^T T)
+size_t layer_scratch(const agzo_layer& a, bool tc, bool long_slabs, bool with_panels = true, int y_parts_min = 0) {
   if (!has_x(a)) return 0;
   int slabs, slab_rows;
   slab_shape(a, tc, long_slabs, &slabs, &slab_rows);
+  if (slabs < y_parts_min) slabs = y_parts_min;
   const size_t r = (size_t)a.r, d = (size_t)a.d_in, m = (size_t)a.m;
   const size_t gch = (d + 127) / 128;
   size_t b = 0;
@@ -330,17 +334,26 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
 
   // extraction waves: consecutive layers whose activations fit the wave budget and whose
   // scratch fits the workspace
-  // layers whose power steps run in the fused kernel keep 2048-token slabs (a slab is that kernel's
-  // work item); the long slabs are for the layers that the two-sweep kernels serve
+  // A layer that shares its X with a neighbour stays with the two-sweep kernels unless fusing is forced: one
+  // sweep serves the whole group there, which moves fewer bytes per layer than one fused pass per layer.
+  auto shares_input = [&](int k) {
+    if (!opts.share_inputs) return false;
+    return (k > 0 && has_x(L[k - 1]) && tc_eligible(L[k - 1]) && same_input(L[k - 1], L[k])) ||
+           (k + 1 < n && has_x(L[k + 1]) && tc_eligible(L[k + 1]) && same_input(L[k], L[k + 1]));
+  };
   auto runs_fused = [&](const agzo_layer& a) {
-    return opts.extract_fused && extract_path != 1 && extract_path != 3 && tc_available && tc_eligible(a) && fused_eligible(a);
+    return opts.extract_fused && extract_path != 1 && extract_path != 3 && tc_available && tc_eligible(a) &&
+           fused_eligible(a, opts.extract_fused == 2) && (opts.extract_fused == 2 || !shares_input((int)(&a - L)));
   };
   long long column_blocks = 0;
   for (int k = 0; k < n; ++k)
-    if (has_x(L[k]) && extract_path != 1 && tc_available && tc_eligible(L[k]) && !runs_fused(L[k]))
+    if (has_x(L[k]) && extract_path != 1 && tc_available && tc_eligible(L[k]))
       column_blocks += (L[k].d_in + 127) / 128;
   const bool long_slabs_any = column_blocks >= kLongSlabColumnBlocks;
-  auto long_slabs_for = [&](const agzo_layer& a) { return long_slabs_any && !runs_fused(a); };
+  auto long_slabs_for = [&](const agzo_layer&) { return long_slabs_any; };
+  auto y_parts_min = [&](const agzo_layer& a) {
+    return runs_fused(a) ? fused_parts_bound(a, fused_cluster_size(a, opts.extract_fused == 2)) : 0;
+  };
   int i = 0;
   while (i < n) {
     if (!has_x(L[i])) {
@@ -370,7 +383,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       }
       auto unit_need = [&](int len, int nrows) {
         size_t b = 0;
-        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, long_slabs_for(L[j + g]), false);
+        for (int g = 0; g < len; ++g) b += layer_scratch(L[j + g], tc, long_slabs_for(L[j + g]), false, y_parts_min(L[j + g]));
         if (tc) b += tc_panel_bytes(L[j], nrows);
         return b;
       };
@@ -397,7 +410,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
           const size_t gch = (d + 127) / 128;
           D.slabs = slabs; D.slab_rows = slab_rows; D.gchunks = (int)gch;
           D.T = reinterpret_cast<float*>(p);      p += align_up(m * r * 4);
-          D.Ypart = reinterpret_cast<float*>(p);  p += align_up((size_t)slabs * r * d * 4);
+          const size_t parts = (size_t)(slabs > y_parts_min(a) ? slabs : y_parts_min(a));
+          D.Ypart = reinterpret_cast<float*>(p);  p += align_up(parts * r * d * 4);
           D.Gpart = reinterpret_cast<double*>(p); p += align_up(gch * r * r * 8);
           D.M = reinterpret_cast<double*>(p);     p += align_up(r * r * 8);
         }
@@ -413,7 +427,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
             D.grp_NB = g == 0 ? rows : 0;
             D.tmaps = ws + maps_offset(n) + (size_t)(j + g) * kMapBytes;
             // the power steps of this layer run fused (X read once per step) where its shape allows
-            D.fz_C = (opts.extract_fused && extract_path != 3 && fused_eligible(a)) ? fused_cluster_size(a) : 0;
+            D.fz_C = runs_fused(a) ? fused_cluster_size(a, opts.extract_fused == 2) : 0;
+            D.fz_slice = fused_slice_cols(a, opts.extract_fused == 2);
           }
         }
       }
@@ -439,6 +454,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       std::stable_sort(ord.begin(), ord.end(), [&](int a, int b) { return L[i + a].d_in > L[i + b].d_in; });
       for (int k = 0; k < j - i; ++k) plan->dev[i + k].xq_order = ord[k];
     }
+    if (ws)   // the fused kernel's launches of this wave, one per cluster size: who works on which tiles
+      for (int C = 1; C <= 16; ++C) fused_plan_shares(plan->dev.data(), i, j, C);
     plan->wave_end.push_back(j);
     plan->wave_region.push_back(region);
     i = j;
@@ -474,7 +491,7 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   if (kHeaderBytes + table_bytes(n) > c->ws_bytes) return AGZO_ERR_WORKSPACE;
   Plan plan;
   PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels, c->rmw_stage_r,
-                c->tc.available, c->extract_fused != 0, c->share_inputs != 0,
+                c->tc.available, c->extract_fused, c->share_inputs != 0,
                 c->allreduce ? 1 : c->extract_streams};   // the ranks' sums run in wave order on the caller's stream
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
@@ -585,9 +602,13 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, false, false, 2}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 0, false, 2}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, false, false, 2}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, 0, false, 2}, &plan, &scratch_cc);
+  if (st != AGZO_OK) return st;
+  if (scratch_cc > scratch) scratch = scratch_cc;
+  // ... and for the fused power step, whose layers keep short token slabs
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 2, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -619,7 +640,7 @@ agzo_status agzo_create(agzo_ctx** out, int device, void* workspace, size_t work
   c->rmw_stage_r = 0;
   c->wave_bytes = kDefaultWaveBytes;
   c->extract_streams = 2;
-  c->extract_fused = 0;
+  c->extract_fused = 1;
   c->allreduce = nullptr;
   c->rimg_valid = false;
   c->rimg_seed = 0;
@@ -711,7 +732,7 @@ agzo_status agzo_set_option(agzo_ctx* ctx, const char* name, int64_t value) {
     if (value < 0 || value > 1) return AGZO_ERR_INVALID_ARG;
     ctx->share_inputs = (int)value;
   } else if (std::strcmp(name, "extract_fused") == 0) {
-    if (value < 0 || value > 1) return AGZO_ERR_INVALID_ARG;
+    if (value < 0 || value > 2) return AGZO_ERR_INVALID_ARG;
     ctx->extract_fused = (int)value;
   } else if (std::strcmp(name, "extract_streams") == 0) {
     if (value < 1 || value > 2) return AGZO_ERR_INVALID_ARG;
@@ -759,6 +780,27 @@ agzo_status agzo_read_counters(agzo_ctx* ctx, double* h_ms, int64_t* h_timed, in
   if (h_total) *h_total = ctx->launches;
   ctx->events_used = 0;
   ctx->launches = 0;
+  return AGZO_OK;
+}
+
+agzo_status agzo_query_cluster_capacity(agzo_ctx* ctx, int32_t* h_clusters) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!h_clusters) return AGZO_ERR_INVALID_ARG;
+  for (int C = 0; C <= 16; ++C) h_clusters[C] = ctx->tc.available ? fused_resident_clusters(C) : 0;
+  return AGZO_OK;
+}
+
+agzo_status agzo_query_fused(agzo_ctx* ctx, const agzo_layer* h_layers, int n, int32_t* h_cluster, void* stream) {
+  agzo_status st = check_ctx(ctx);
+  if (st != AGZO_OK) return st;
+  if (!h_cluster || n < 0) return AGZO_ERR_INVALID_ARG;
+  st = validate(h_layers, n, 0);
+  if (st != AGZO_OK) return st;
+  if (n == 0) return AGZO_OK;
+  st = prepare(ctx, h_layers, n, static_cast<cudaStream_t>(stream));
+  if (st != AGZO_OK) return st;
+  for (int i = 0; i < n; ++i) h_cluster[i] = ctx->plan.dev[i].fz_C;
   return AGZO_OK;
 }
 
@@ -858,10 +900,10 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
         return all_tc ? tc_x_q(ctx->tc, w, P.dev.data(), dst, true, ws) : launch_x_q(w, ws);
       };
       auto power_fused = [&]() -> cudaError_t {              // Y <- H (H^T Q) in one pass
-        for (int C = 1; C <= 8; ++C) {
+        for (int C = 1; C <= 16; ++C) {
           if (!(fz_classes & (1u << C))) continue;
           Timed t(ctx, AGZO_KC_FUSED_POWER, ws);
-          cudaError_t e = launch_fused_power_step(w, P.dev.data(), C, dst, ctx->sm_count, ws);
+          cudaError_t e = launch_fused_power_step(w, P.dev.data(), C, dst, ws);
           if (e != cudaSuccess) return e;
         }
         return cudaSuccess;
@@ -872,7 +914,10 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
       for (int k = 0; k < K; ++k) {
         if ((sr = sum_over_ranks()) != AGZO_OK) return sr;
         CU(ctx, panel_qr());                   // Q <- qr(Y)
-        if (fz_classes) CU(ctx, power_fused());
+        if (fz_classes) {
+          CU(ctx, power_fused());
+          w.after_fused = 1;                   // their partial sums are now one per share, not one per slab
+        }
         if (any_unfused) {
           CU(ctx, x_q());
           CU(ctx, xt_t(true));                 // Y <- H (H^T Q)

@@ -40,6 +40,13 @@ struct alignas(16) DevLayer {
   int NB, NP;
   int xq_order;          // T = X Q: the CTA row of this wave position works on layer (wave start + xq_order), longest rows first
   int fz_C;              // cluster size of the fused power-step kernel for this layer, 0 = unfused kernels
+  int fz_slice;          // columns of X per CTA of that cluster
+  // The fused kernel's launch for the wave's layers of one cluster size treats their 128-token tiles as one
+  // list, cut into equal contiguous shares, one per cluster; a share that ends inside a layer leaves a
+  // partial Y for it, so a layer has as many partial sums (in Ypart) as clusters whose shares meet it.
+  int fz_tile0;          // index of this layer's first tile in that list
+  int fz_first;          // the first share that meets this layer
+  int fz_parts;          // partial sums of this layer after a fused power step
   // Consecutive layers that read the same X (q/k/v, gate/up of a transformer block) form a group:
   // their operand panels are adjacent rows of one matrix, the leader's CTAs run both products
   // for all members with N = grp_NB columns, and X is read once per product for the group.
@@ -155,7 +162,13 @@ struct ExtractWave {
   int max_m, max_din, max_r, max_slabs, max_gchunks;
   long long omega_row0;       // global index of the first local token (token-sharded extraction), else 0
   int y_reduced;              // 1: Y already holds the sum over slabs (and ranks); the panel QR reads it as it is
+  int after_fused;            // 1: the last product was a power step, so the layers of the fused kernel have
+                              // fz_parts partial sums in Ypart (the others, and everyone after X^T T: slabs)
 };
+// number of partial sums of Y that the layer's last product left in Ypart
+__host__ __device__ inline int y_parts(const DevLayer& L, int after_fused) {
+  return (after_fused && L.fz_C) ? L.fz_parts : L.slabs;
+}
 cudaError_t launch_fill_omega(const ExtractWave& w, uint64_t seed, cudaStream_t s);
 cudaError_t launch_xt_t(const ExtractWave& w, cudaStream_t s);      // Ypart = X^T T per slab
 cudaError_t launch_x_q(const ExtractWave& w, cudaStream_t s);       // T = X Q (Q read from V)

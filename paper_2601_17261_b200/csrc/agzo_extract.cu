@@ -182,8 +182,10 @@ inline size_t gram_smem_bytes_upto(int max_r) {
   for (int r = 1; r <= max_r; ++r) b = gram_smem_bytes(r) > b ? gram_smem_bytes(r) : b;
   return b;
 }
-__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0, int y_reduced) {
+__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0, int y_reduced,
+                                                          int after_fused) {
   const DevLayer& L = layers[l0 + blockIdx.y];
+  const int nparts = y_parts(L, after_fused);
   const int ngroups = (L.gchunks + kGramGroup - 1) / kGramGroup;
   const int grp = blockIdx.x;
   if (grp >= ngroups) return;
@@ -214,7 +216,7 @@ __global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __rest
         if (y_reduced) {
           y = L.Y[(long long)k * L.d_in + d];
         } else {
-          for (int s = 0; s < L.slabs; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
+          for (int s = 0; s < nparts; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
           L.Y[(long long)k * L.d_in + d] = y;
         }
       }
@@ -399,12 +401,13 @@ __global__ void __launch_bounds__(128) apply_kernel(const DevLayer* __restrict__
 
 // Y[k][d] = sum_s Ypart[s][k][d] in slab order, on its own: token-sharded extraction sums Y over
 // the ranks before the panel QR reads it
-__global__ void __launch_bounds__(256) sum_slabs_kernel(const DevLayer* __restrict__ layers, int l0) {
+__global__ void __launch_bounds__(256) sum_slabs_kernel(const DevLayer* __restrict__ layers, int l0, int after_fused) {
   const DevLayer& L = layers[l0 + blockIdx.y];
+  const int nparts = y_parts(L, after_fused);
   const long long n = (long long)L.r * L.d_in;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
     float y = 0.f;
-    for (int s = 0; s < L.slabs; ++s) y += L.Ypart[(long long)s * n + i];
+    for (int s = 0; s < nparts; ++s) y += L.Ypart[(long long)s * n + i];
     L.Y[i] = y;
   }
 }
@@ -412,14 +415,14 @@ __global__ void __launch_bounds__(256) sum_slabs_kernel(const DevLayer* __restri
 cudaError_t launch_sum_slabs(const ExtractWave& w, cudaStream_t s) {
   long long blocks = ((long long)w.max_r * w.max_din + 255) / 256;
   if (blocks > 256) blocks = 256;
-  sum_slabs_kernel<<<dim3((unsigned)blocks, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0);
+  sum_slabs_kernel<<<dim3((unsigned)blocks, w.l1 - w.l0), 256, 0, s>>>(w.d_layers, w.l0, w.after_fused);
   return cudaGetLastError();
 }
 
 cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s) {
   const int nl = w.l1 - w.l0;
   reduce_gram_kernel<<<dim3((w.max_gchunks + kGramGroup - 1) / kGramGroup, nl), 256, gram_smem_bytes_upto(w.max_r), s>>>(
-      w.d_layers, w.l0, w.y_reduced);
+      w.d_layers, w.l0, w.y_reduced, w.after_fused);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t chol_bytes = chol_smem_bytes(w.max_r);

@@ -3,22 +3,23 @@
 // The two products of a power step meet the same X: T = X Q needs a whole row of X (all of d_in)
 // before a single element of Y = X^T T can be formed, so the unfused kernels read X twice from
 // HBM.  Here a thread-block cluster of C CTAs shares a tile of 128 tokens; CTA c works on its
-// 512-column slice of the tile:
-//   phase A   the slice's contribution to T (128 x NB, tcgen05.mma M = 128, K = 512) goes to TMEM;
+// slice of the tile's columns (512 of them in clusters of up to 16; 768 where d_in is beyond 16 x 512):
+//   phase A   the slice's contribution to T (128 x NB, tcgen05.mma M = 128) goes to TMEM;
 //             X streams through a ring of shared-memory slots (first read, from HBM, marked
 //             evict-last for L2) and every slot is released as soon as its MMAs have read it,
 //   exchange  the C partial sums are added up through distributed shared memory in two one-way
 //             hops (st.async): groups of eight token rows are summed in rank order by the CTA that
 //             owns them, which writes the bf16 hi/lo parts of the sums straight into the T operand
 //             buffer of every CTA of the cluster,
-//   phase C   Y_slice (512 x NB, kept in TMEM across all tiles of the work item) += X_slice^T T;
+//   phase C   Y_slice (slice x NB, kept in TMEM across all tiles of the work item) += X_slice^T T;
 //             the slice is fetched a second time through a second, smaller ring -- a few boxes
 //             behind the first read, so it comes from L2 (measured: a line survives 20 to 50 MB of
 //             streaming traffic, and this lag is about one tile per CTA).
 // An earlier version kept the tile resident in shared memory between the phases; the exchange
 // takes about 2 us, the ring held 2.5 tiles of 64 KiB, and that residency, not the arithmetic,
-// bounded it at 3.6 TB/s.  A work item is (layer, token slab); the slab's partial Y leaves TMEM
-// once, at the end of the item, and the slabs are summed by the panel QR.
+// bounded it at 3.6 TB/s.  The tiles of all layers of a launch form one list that is cut into equal
+// contiguous shares, one per cluster; where a share ends inside a layer the partial Y leaves TMEM for
+// that layer's next partial-sum buffer, and the panel QR adds a layer's partial sums in share order.
 //
 // As in the unfused kernels Q and T are fp32 quantities carried as hi + lo bf16 pairs in NB = 2 NP
 // operand columns (NP = r rounded up to 8), products exact, accumulation fp32.
@@ -44,18 +45,18 @@ constexpr int kFzThreads = 11 * 32;        // producer A, MMA, two epilogue grou
 constexpr int kWarpProdC = 10;
 constexpr int kTT = 128;                   // tokens per tile
 constexpr int kGroups = kTT / 8;           // token groups of a tile (the unit of ownership in the exchange)
-constexpr int kSliceCols = 512;            // columns of X per CTA
-constexpr int kMBlocks = kSliceCols / 128; // M blocks of phase C
+constexpr int kSliceCols = 512;            // columns of X per CTA ...
+constexpr int kWideSliceCols = 768;        // ... and where 16 such slices do not cover d_in
+constexpr int kMaxCluster = 16;
 constexpr int kSlotBytes = 16 * 1024;      // ring A: [128 tokens][64 columns]; ring C: [64 tokens][128 columns]
 constexpr int kBoxBytes = 8 * 1024;        // one TMA box of 64 tokens x 64 columns
-constexpr int kRingA = 5, kRingC = 4;
+constexpr int kRingC = 4;                  // ring A: 5 slots, 4 beside the Q region of a wide slice
 constexpr int kMaxRing = 8;
 constexpr int kLook = 2;                   // phase A runs up to this many tiles ahead of phase C
 constexpr int kBuf = kLook + 1;            // T partial (TMEM) and T operand (shared memory) buffers in rotation
 constexpr int kRs = 2;                     // exchange buffers in rotation
 constexpr int kRsFloats = 2688;            // C * ceil(16 / C) * 8 * NP floats at most (C = 7, NP = 16)
 constexpr int kTtBytes = 32 * 256;         // T operand: up to 32 rows of 128 tokens
-constexpr uint32_t kFzTmemCols = 256;
 
 struct FzShared {
   uint64_t xa_full[kMaxRing], xa_empty[kMaxRing];
@@ -69,53 +70,76 @@ struct FzShared {
   int failed;
 };
 
+// One piece of a cluster's share: tiles of a layer from token t_begin on, whose sum goes to the layer's
+// partial Y number `part`.
 struct FzItem {
   const DevLayer* L;
-  int slab, t_begin, ntiles;
+  int part, t_begin, ntiles;
 };
 
-// item -> (layer, slab) among the layers of [l0, l1) whose cluster size is C; false past the end
-__device__ __forceinline__ bool fz_decode(const DevLayer* layers, int l0, int l1, int C, int item, FzItem* it) {
-  for (int l = l0; l < l1; ++l) {
-    const DevLayer* L = layers + l;
-    if (L->fz_C != C) continue;
-    if (item < L->slabs) {
+// `total` tiles cut into G shares: the first `rem` shares have base + 1 tiles, the others base
+// (base = total / G, rem = total % G, both worked out on the host: the kernel divides nothing).
+__host__ __device__ inline int fz_share_begin(int k, int base, int rem) { return k * base + (k < rem ? k : rem); }
+inline int fz_share_of(int off, int base, int rem) {      // the share that holds tile `off`
+  const int big = rem * (base + 1);
+  return off < big ? off / (base + 1) : rem + (off - big) / base;
+}
+
+// Walks the pieces of this cluster's share: the layers of [l0, l1) with cluster size C in order, their tiles
+// as one list.  A layer's pieces are numbered from the first share that meets it (fz_first).
+struct FzWalk {
+  int l, lo, hi;      // next layer to look at; the share's tile range
+  __device__ FzWalk(int l0, int cluster, int base, int rem)
+      : l(l0), lo(fz_share_begin(cluster, base, rem)), hi(fz_share_begin(cluster + 1, base, rem)) {}
+  __device__ bool next(const DevLayer* layers, int l1, int C, int cluster, FzItem* it) {
+    for (; l < l1; ++l) {
+      const DevLayer* L = layers + l;
+      if (L->fz_C != C) continue;
+      const int nt = (L->m + kTT - 1) / kTT;
+      const int b = max(lo, L->fz_tile0), e = min(hi, L->fz_tile0 + nt);
+      if (b >= e) continue;
       it->L = L;
-      it->slab = item;
-      it->t_begin = item * L->slab_rows;
-      const int t_end = min(L->m, it->t_begin + L->slab_rows);
-      it->ntiles = (t_end - it->t_begin + kTT - 1) / kTT;
+      it->part = cluster - L->fz_first;
+      it->t_begin = (b - L->fz_tile0) * kTT;
+      it->ntiles = e - b;
+      ++l;
       return true;
     }
-    item -= L->slabs;
+    return false;
   }
-  return false;
-}
+};
 
 __device__ __forceinline__ uint32_t swz(int i, int j) {
   return (uint32_t)((i >> 3) * 1024 + (i & 7) * 128 + ((j ^ (i & 7)) << 4));
 }
 
+// kWide: some layer of the launch has 768-column slices (its Q slice takes 12 boxes instead of 8, so ring A
+// has one slot less, and its six Y accumulators need more than 256 TMEM columns) or the cluster has more
+// than 8 CTAs.  Two instantiations, because only the wide one is marked for cluster sizes beyond the
+// portable 8.
+template <bool kWide>
 __global__ void __launch_bounds__(kFzThreads, 1)
-fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, DevStatus* status) {
+fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, int share_base, int share_rem,
+                        DevStatus* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ FzShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();
-  const int cluster = (int)cluster_id_x(), nclusters = (int)cluster_count_x();
-  const int col0 = rank * kSliceCols;
-  // shared-memory carve-up: ring A | ring C | Q slice (8 boxes of [NB][64]) | T operand x kBuf | exchange buffers x kRs | staging
+  const int cluster = (int)cluster_id_x();
+  constexpr int ring_a = kWide ? 4 : 5;
+  constexpr uint32_t tmem_cols = kWide ? 512u : 256u;
+  // shared-memory carve-up: ring A | ring C | Q slice (boxes of [NB][64]) | T operand x kBuf | exchange buffers x kRs | staging
   uint8_t* sXA = base;
-  uint8_t* sXC = sXA + (size_t)kRingA * kSlotBytes;
+  uint8_t* sXC = sXA + (size_t)ring_a * kSlotBytes;
   uint8_t* sQ = sXC + (size_t)kRingC * kSlotBytes;
   // NB is a per-layer quantity; the regions are sized for NB = 32
-  uint8_t* sTt = sQ + 8 * 32 * 128;
+  uint8_t* sTt = sQ + (kWide ? 12 : 8) * 32 * 128;
   float* sRs = reinterpret_cast<float*>(sTt + kBuf * kTtBytes);   // kRs x [C][cpo][8][NP] floats
   uint8_t* sStage = reinterpret_cast<uint8_t*>(sRs + kRs * kRsFloats);   // 512 bytes per epilogue warp
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kRingA; ++s) { mbar_init(&sh.xa_full[s], 1); mbar_init(&sh.xa_empty[s], 1); }
+    for (int s = 0; s < ring_a; ++s) { mbar_init(&sh.xa_full[s], 1); mbar_init(&sh.xa_empty[s], 1); }
     for (int s = 0; s < kRingC; ++s) { mbar_init(&sh.xc_full[s], 1); mbar_init(&sh.xc_empty[s], 1); }
     mbar_init(&sh.qb_full, 1); mbar_init(&sh.qb_empty, 1);
     for (int p = 0; p < kBuf; ++p) {
@@ -128,7 +152,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
   }
-  if (warp == 1) tmem_alloc(&sh.tmem_base, kFzTmemCols);
+  if (warp == 1) tmem_alloc(&sh.tmem_base, tmem_cols);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();          // every CTA's barriers exist before anyone arrives on them remotely
@@ -142,14 +166,15 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       int ns = 0, ic = 0;
       bool ok = true;
       FzItem it;
-      for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters, ++ic) {
+      for (FzWalk walk(l0, cluster, share_base, share_rem); ok && walk.next(layers, l1, C, cluster, &it); ++ic) {
         const DevLayer& L = *it.L;
         const uint8_t* maps = reinterpret_cast<const uint8_t*>(L.tmaps);
         const void* map_x = maps;
         const void* map_q = maps + 128;
         tmap_acquire(map_x);
         tmap_acquire(map_q);
-        const int live = min(kSliceCols, L.d_in - col0);
+        const int col0 = rank * L.fz_slice;
+        const int live = min(L.fz_slice, L.d_in - col0);
         const int nq = (live + 63) / 64;                 // live 64-column boxes of this slice
         const int q_box = L.NB * 128;
         if (ic > 0 && !mbar_wait(&sh.qb_empty, (ic - 1) & 1)) { ok = false; break; }
@@ -158,7 +183,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
         for (int tile = 0; tile < it.ntiles && ok; ++tile) {
           const int t0 = it.t_begin + tile * kTT;
           for (int j = 0; j < nq; ++j, ++ns) {
-            const int s = ns % kRingA, u = ns / kRingA;
+            const int s = ns % ring_a, u = ns / ring_a;
             if (u > 0 && !mbar_wait(&sh.xa_empty[s], (u - 1) & 1)) { ok = false; break; }
             uint8_t* slot = sXA + (size_t)s * kSlotBytes;
             mbar_expect_tx(&sh.xa_full[s], kSlotBytes);
@@ -169,7 +194,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       }
       if (!ok) sh.failed = 1;
       if (!ok || sh.failed) {   // leaving early: the copies in flight must land before the CTA goes away
-        for (int k = ns > kRingA ? ns - kRingA : 0; k < ns; ++k) mbar_wait(&sh.xa_full[k % kRingA], (k / kRingA) & 1);
+        for (int k = ns > ring_a ? ns - ring_a : 0; k < ns; ++k) mbar_wait(&sh.xa_full[k % ring_a], (k / ring_a) & 1);
       }
     }
   } else if (warp == kWarpProdC) {
@@ -179,11 +204,12 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       int ns = 0;
       bool ok = true;
       FzItem it;
-      for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters) {
+      for (FzWalk walk(l0, cluster, share_base, share_rem); ok && walk.next(layers, l1, C, cluster, &it); ) {
         const DevLayer& L = *it.L;
         const void* map_x = L.tmaps;
         tmap_acquire(map_x);
-        const int live = min(kSliceCols, L.d_in - col0);
+        const int col0 = rank * L.fz_slice;
+        const int live = min(L.fz_slice, L.d_in - col0);
         const int mb = (live + 127) / 128;               // live M blocks
         for (int tile = 0; tile < it.ntiles && ok; ++tile) {
           const int t0 = it.t_begin + tile * kTT;
@@ -216,15 +242,16 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       bool ok = true;
       FzItem it;
       const uint32_t sq_addr = smem_u32(sQ), sxa_addr = smem_u32(sXA), sxc_addr = smem_u32(sXC), stt_addr = smem_u32(sTt);
-      for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters, ++ic) {
+      for (FzWalk walk(l0, cluster, share_base, share_rem); ok && walk.next(layers, l1, C, cluster, &it); ++ic) {
         const DevLayer& L = *it.L;
         const int NB = L.NB;
-        const int live = min(kSliceCols, L.d_in - col0);
+        const int col0 = rank * L.fz_slice;
+        const int live = min(L.fz_slice, L.d_in - col0);
         const int nq = (live + 63) / 64, mb = (live + 127) / 128;
         const uint32_t q_box = (uint32_t)NB * 128u;
         const uint32_t idesc_a = instr_desc(128, NB, 0, 0);
         const uint32_t idesc_c = instr_desc(128, NB, 1, 0);      // A = X boxes read as X^T
-        const uint32_t tp_col = (uint32_t)(kMBlocks * NB);       // T partials sit after the Y accumulators
+        const uint32_t tp_col = (uint32_t)((L.fz_slice / 128) * NB);   // T partials sit after the Y accumulators
         if (!mbar_wait_warp(&sh.qb_full, ic & 1)) { ok = false; break; }
         if (ic > 0 && !mbar_wait_warp(&sh.y_free, (ic - 1) & 1)) { ok = false; break; }
         // The two phases are issued as their operands arrive, whichever is ready: phase A of tile a_tile box by
@@ -244,7 +271,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
           if (a_tile < it.ntiles && (a_tile <= c_tile + 1 || (a_tile == c_tile + 2 && tt_ready))) {
             const int p = ta % kBuf, u2 = ta / kBuf;
             if (a_box == 0 && u2 > 0 && !mbar_wait_warp(&sh.tp_empty[p], (u2 - 1) & 1)) { ok = false; break; }
-            const int s = na % kRingA, u = na / kRingA;
+            const int s = na % ring_a, u = na / ring_a;
             if (mbar_test_warp(&sh.xa_full[s], u & 1)) {
               tc_fence_after();
               const uint32_t d_tp = tmem + tp_col + (uint32_t)(p * NB);
@@ -315,12 +342,13 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
     int te = 0, ic = 0;
     bool ok = true;
     FzItem it;
-    for (int item = cluster; ok && fz_decode(layers, l0, l1, C, item, &it); item += nclusters, ++ic) {
+    for (FzWalk walk(l0, cluster, share_base, share_rem); ok && walk.next(layers, l1, C, cluster, &it); ++ic) {
       const DevLayer& L = *it.L;
       const int NB = L.NB, NP = L.NP, r = L.r;
-      const int live = min(kSliceCols, L.d_in - col0);
+      const int col0 = rank * L.fz_slice;
+      const int live = min(L.fz_slice, L.d_in - col0);
       const int mb = (live + 127) / 128;
-      const uint32_t tp_col = (uint32_t)(kMBlocks * NB);
+      const uint32_t tp_col = (uint32_t)((L.fz_slice / 128) * NB);
       const int cpo = (kGroups + C - 1) / C;   // token groups of a tile per owner, at most
       for (int tile = 0; tile < it.ntiles && ok; ++tile, ++te) {
         const int p = te % kBuf, u2 = te / kBuf;     // T partial and T operand buffers
@@ -429,7 +457,7 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
       tc_fence_after();
       for (int b = 0; b < mb; ++b) {
         const int d = col0 + b * 128 + q * 32 + lane;
-        float* out = L.Ypart + (long long)it.slab * r * L.d_in + d;
+        float* out = L.Ypart + (long long)it.part * r * L.d_in + d;
         for (int k0 = 0; k0 < NP; k0 += 8) {
           float hi[8], lo[8];
           tmem_ld8(tmem + lane_off + (uint32_t)(b * NB + k0), hi);
@@ -451,37 +479,19 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
   __syncthreads();
   if (sh.failed && threadIdx.x == 0) { atomicExch(&status->timeout, 1); atomicExch(&status->where, 4); }
   cluster_sync_all();          // no peer reads my exchange buffer or arrives on my barriers after this
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, kFzTmemCols); }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, tmem_cols); }
 }
 
-int g_max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // per cluster size, filled on first use
+// Clusters of this kernel that can be resident at once, per cluster size; filled by fused_init (a cluster
+// has to fit into one GPC, so sizes that do not divide a GPC's SMs leave part of the device idle).
+int g_max_clusters[2][kMaxCluster + 1] = {};   // [narrow / wide instantiation][cluster size]
+int g_sm_count = 0;                         // 0 until fused_init has run
 
 size_t fz_smem_bytes() {
-  return (size_t)(kRingA + kRingC) * kSlotBytes + 8 * 32 * 128 + kBuf * kTtBytes + kRs * kRsFloats * 4 + 8 * 512 + 1024;
+  return (size_t)(5 + kRingC) * kSlotBytes + 8 * 32 * 128 + kBuf * kTtBytes + kRs * kRsFloats * 4 + 8 * 512 + 1024;
 }
 
-}  // namespace
-
-bool fused_eligible(const agzo_layer& a) {
-  return tc_eligible(a) && a.r <= 16 && a.d_in <= 8 * kSliceCols && a.m >= kTT;
-}
-
-int fused_cluster_size(const agzo_layer& a) { return (a.d_in + kSliceCols - 1) / kSliceCols; }
-
-cudaError_t fused_init() {
-  cudaError_t e = cudaFuncSetAttribute(fused_power_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)fz_smem_bytes());
-  return e;
-}
-
-// One fused power step for the layers of the wave whose cluster size is C.
-cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
-                                    int sm_count, cudaStream_t s) {
-  int items = 0;
-  for (int i = w.l0; i < w.l1; ++i)
-    if (h_dev[i].fz_C == C) items += h_dev[i].slabs;
-  if (items == 0) return cudaSuccess;
-  const size_t smem = fz_smem_bytes();
+cudaError_t fz_max_clusters(bool wide, int C, int sm_count, int* n) {
   cudaLaunchConfig_t cfg{};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -489,25 +499,140 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.blockDim = dim3(kFzThreads);
-  cfg.dynamicSmemBytes = smem;
+  cfg.gridDim = dim3((unsigned)(C * (sm_count / C)));
+  cfg.dynamicSmemBytes = fz_smem_bytes();
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return wide ? cudaOccupancyMaxActiveClusters(n, fused_power_step_kernel<true>, &cfg)
+              : cudaOccupancyMaxActiveClusters(n, fused_power_step_kernel<false>, &cfg);
+}
+
+}  // namespace
+
+// The slice width of a layer: 512 or 768 columns, among those with which the cluster has at most 16 CTAs and
+// the exchange buffer of the busiest owner (C sources x its token groups x 8 tokens x NP sums) fits.  A
+// cluster has to fit into one GPC, so some sizes leave SMs idle, and the last slice of a layer may be
+// partly empty: what counts is the share of the device's SM-time that works on columns of X,
+//   (d_in / slice) x resident clusters / SMs.
+// The width with the larger share wins (512 on a tie), and below 70 % the layer is left to the two sweeps
+// of the unfused kernels, which are faster then; 0 when neither width qualifies.  Before fused_init has
+// run (sizing a workspace without a device) the shape alone decides; with any_size the 70 % rule is
+// dropped (every cluster size that the device can launch at all).
+int fused_slice_cols(const agzo_layer& a, bool any_size) {
+  const int NP = (a.r + 7) / 8 * 8;
+  int best = 0;
+  double best_share = -1.0;
+  for (int slice : {kSliceCols, kWideSliceCols}) {
+    const int C = (a.d_in + slice - 1) / slice;
+    if (C > kMaxCluster) continue;
+    if (C * ((kGroups + C - 1) / C) * 8 * NP > kRsFloats) continue;
+    double share = 0.0;
+    if (g_sm_count) {
+      const int resident = g_max_clusters[slice > kSliceCols || C > 8][C];
+      if (resident <= 0) continue;
+      share = (double)a.d_in / slice * resident / g_sm_count;
+      if (!any_size && share < 0.7) continue;
+    }
+    if (share > best_share) { best = slice; best_share = share; }
+  }
+  return best;
+}
+
+int fused_cluster_size(const agzo_layer& a, bool any_size) {
+  const int slice = fused_slice_cols(a, any_size);
+  return slice ? (a.d_in + slice - 1) / slice : 0;
+}
+
+bool fused_eligible(const agzo_layer& a, bool any_size) {
+  return tc_eligible(a) && a.r <= 16 && a.m >= kTT && fused_slice_cols(a, any_size) != 0;
+}
+
+cudaError_t fused_init(int sm_count) {
+  cudaError_t e = cudaFuncSetAttribute(fused_power_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)fz_smem_bytes());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fused_power_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)fz_smem_bytes());
+  if (e != cudaSuccess) return e;
+  // clusters of more than 8 CTAs are beyond the portable size: ask for them, and use them only if they fit
+  const bool big = cudaFuncSetAttribute(fused_power_step_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed,
+                                        1) == cudaSuccess;
+  for (int C = 1; C <= kMaxCluster; ++C) {
+    int n = 0;
+    if (C > 8 || fz_max_clusters(false, C, sm_count, &n) != cudaSuccess) n = 0;
+    g_max_clusters[0][C] = n;
+    n = 0;
+    if ((C > 8 && !big) || fz_max_clusters(true, C, sm_count, &n) != cudaSuccess) n = 0;
+    g_max_clusters[1][C] = n;
+  }
+  cudaGetLastError();
+  g_sm_count = sm_count;
+  return cudaSuccess;
+}
+
+int fused_resident_clusters(int C) { return C >= 1 && C <= kMaxCluster ? g_max_clusters[C > 8][C] : 0; }
+
+// The partial sums of Y that a fused power step can leave for a layer, at most: one per share that meets it.
+int fused_parts_bound(const agzo_layer& a, int C) {
+  const int nt = (a.m + kTT - 1) / kTT;
+  const int shares = 160 / C;      // no device this kernel runs on has more SMs than that
+  return nt < shares ? nt : shares;
+}
+
+// Cuts the tiles of the layers of [l0, l1) with cluster size C into shares: fills fz_tile0 and fz_parts.
+void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
+  int total = 0;
+  bool wide = C > 8;
+  for (int i = l0; i < l1; ++i)
+    if (dev[i].fz_C == C) {
+      dev[i].fz_tile0 = total;
+      total += (dev[i].m + kTT - 1) / kTT;
+      wide = wide || dev[i].fz_slice > kSliceCols;
+    }
+  if (total == 0) return;
+  const int cap = g_max_clusters[wide][C] > 0 ? g_max_clusters[wide][C] : 1;
+  const int G = total < cap ? total : cap;
+  const int base = total / G, rem = total % G;
+  for (int i = l0; i < l1; ++i)
+    if (dev[i].fz_C == C) {
+      const int nt = (dev[i].m + kTT - 1) / kTT;
+      dev[i].fz_first = fz_share_of(dev[i].fz_tile0, base, rem);
+      dev[i].fz_parts = fz_share_of(dev[i].fz_tile0 + nt - 1, base, rem) - dev[i].fz_first + 1;
+    }
+}
+
+// One fused power step for the layers of the wave whose cluster size is C.
+cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
+                                    cudaStream_t s) {
+  int total = 0;
+  bool wide = C > 8;
+  for (int i = w.l0; i < w.l1; ++i)
+    if (h_dev[i].fz_C == C) {
+      total += (h_dev[i].m + kTT - 1) / kTT;
+      if (h_dev[i].fz_slice > kSliceCols) wide = true;
+    }
+  if (total == 0) return cudaSuccess;
+  if (C < 1 || C > kMaxCluster || g_max_clusters[wide][C] <= 0) return cudaErrorInvalidConfiguration;   // the planner picks no such size
+  cudaLaunchConfig_t cfg{};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(kFzThreads);
+  cfg.dynamicSmemBytes = fz_smem_bytes();
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (g_max_clusters[C] == 0) {
-    cfg.gridDim = dim3((unsigned)(C * (sm_count / C)));
-    int n = 0;
-    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, fused_power_step_kernel, &cfg);
-    if (e != cudaSuccess) return e;
-    g_max_clusters[C] = n > 0 ? n : 1;
-  }
-  // persistent clusters: never more than can be resident at once (they wait on one another only
-  // inside a cluster, but a resident set keeps the schedule static)
-  const int nclusters = items < g_max_clusters[C] ? items : g_max_clusters[C];
+  // persistent clusters, never more than can be resident at once; the same count as fused_plan_shares used
+  const int nclusters = total < g_max_clusters[wide][C] ? total : g_max_clusters[wide][C];
   cfg.gridDim = dim3((unsigned)(nclusters * C));
   const DevLayer* layers = w.d_layers;
   int l0 = w.l0, l1 = w.l1;
-  void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&d_status};
-  return cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel, args);
+  int base = total / nclusters, rem = total % nclusters;
+  void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&base, (void*)&rem, (void*)&d_status};
+  return wide ? cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel<true>, args)
+                         : cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel<false>, args);
 }
 
 }  // namespace agzo

@@ -415,7 +415,11 @@ cudaError_t tc_init(TcState* st, int device) {
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(tc_xt_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = rmw_tc_init();
-    if (e == cudaSuccess) e = fused_init();
+    if (e == cudaSuccess) {
+      int sms = 0;
+      e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+      if (e == cudaSuccess) e = fused_init(sms);
+    }
     if (e != cudaSuccess) { cudaGetLastError(); st->available = false; }
   }
   return cudaSuccess;

@@ -55,10 +55,15 @@ cudaError_t tc_x_q(const TcState& st, const ExtractWave& w, const DevLayer* h_de
                    DevStatus* d_status, bool skip_fused, cudaStream_t s);
 
 // ---- fused power step (agzo_extract_fused.cu): Y = X^T (X Q) in one pass over X
-bool fused_eligible(const agzo_layer& a);
-int fused_cluster_size(const agzo_layer& a);
-cudaError_t fused_init();
+// any_size: also cluster sizes that leave more than 30 % of the SMs idle
+bool fused_eligible(const agzo_layer& a, bool any_size);
+int fused_cluster_size(const agzo_layer& a, bool any_size);
+int fused_slice_cols(const agzo_layer& a, bool any_size);   // columns of X per CTA of the cluster, 0 = not eligible
+int fused_parts_bound(const agzo_layer& a, int C);              // partial sums of Y a power step can leave, at most
+void fused_plan_shares(DevLayer* dev, int l0, int l1, int C);   // fills fz_tile0 / fz_parts of a wave's layers of size C
+int fused_resident_clusters(int C);                             // clusters of C CTAs the device holds at once (after fused_init)
+cudaError_t fused_init(int sm_count);          // asks the device which cluster sizes fit; eligibility follows it
 cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
-                                    int sm_count, cudaStream_t s);
+                                    cudaStream_t s);
 
 }  // namespace agzo

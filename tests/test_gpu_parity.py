@@ -338,6 +338,12 @@ EXTRACT_CASES = [
     (1024, 4096, 16, 2, 32, True, 2),    # fused power step, clusters of 8
     (1536, 2048, 8, 3, 32, True, 2),     # clusters of 4
     (900, 136, 3, 2, 8, True, 2),        # a single CTA per cluster, ragged token tile
+    (640, 5000, 8, 2, 32, True, 2),      # clusters of 10 (beyond the portable size), ragged last slice
+    (400, 8192, 16, 2, 32, True, 2),     # clusters of 16, 512-column slices
+    (384, 12288, 16, 2, 32, True, 2),    # clusters of 16, 768-column slices
+    (520, 9000, 4, 2, 32, True, 2),      # clusters of 12 on 768-column slices, the last one partly filled
+    (512, 6144, 16, 2, 32, True, 2),     # 12 slices of 512 would overflow the exchange buffer at r = 16: 8 of 768
+    (512, 6144, 8, 2, 32, True, 2),      # 8 slices of 768 keep more SMs busy than 12 of 512
     # the same tensor-core products without the fused power step (two sweeps over X per step)
     (2048, 1024, 8, 3, 32, True, 3),
     (700, 520, 8, 3, 16, True, 3),
@@ -353,7 +359,7 @@ def _run_extract(X, r, K, seed, layer_id, path, x_bf16, pitch=None):
     layers = [B.make_layer(X=Xd, V=Vv, r=r, layer_id=layer_id)]
     with Ctx(layers) as ctx:
         B.agzo_set_option(ctx, "extract_path", path)
-        B.agzo_set_option(ctx, "extract_fused", 1 if path == 2 else 0)
+        B.agzo_set_option(ctx, "extract_fused", 2 if path == 2 else 0)
         B.agzo_extract_subspace(ctx, layers, seed, K)
         st = B.agzo_poll(ctx)
     assert bool((Vd[0] == 7).all() and (Vd[-1] == 7).all() and (Vd[:, X.shape[1]:] == 7).all())
@@ -405,7 +411,7 @@ def test_extract_wave_mixes_fused_and_unfused_layers():
         layers.append(B.make_layer(X=Xd, V=Vd, r=r, layer_id=i))
     with Ctx(layers) as ctx:
         B.agzo_set_option(ctx, "extract_path", 2)
-        B.agzo_set_option(ctx, "extract_fused", 1)
+        B.agzo_set_option(ctx, "extract_fused", 2)
         B.agzo_extract_subspace(ctx, layers, 5, 3)
         assert B.agzo_poll(ctx) == B.AGZO_OK
     for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):

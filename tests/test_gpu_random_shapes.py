@@ -75,7 +75,7 @@ def test_extraction_on_random_shapes(seed0):
         what = dict(specs=specs, K=K, path=path, share=share)
         with Ctx(layers) as ctx:
             B.agzo_set_option(ctx, "extract_path", path)
-            B.agzo_set_option(ctx, "extract_fused", 1 if path == 2 else 0)   # path 2: fused power steps where shapes allow
+            B.agzo_set_option(ctx, "extract_fused", 2 if path == 2 else 0)   # path 2: fused power steps where shapes allow
             B.agzo_set_option(ctx, "share_inputs", share)
             if rng.random() < 0.3:
                 B.agzo_set_option(ctx, "wave_bytes", int(rng.integers(1, 8)) << 20)
