@@ -146,8 +146,9 @@ agzo_status agzo_destroy(agzo_ctx* ctx);
  * ceil(d_in / 512) CTAs, or ceil(d_in / 768)), where that cluster size keeps at least 70 % of
  * the device's SMs busy; 2 = the same without the last condition (every cluster size
  * the device can launch) and also for layers that share their X with a neighbour (with 1 those
- * stay with the sweeps that serve the whole group); 0 = off: two sweeps over X per power step.
- * Default 1;
+ * stay with the sweeps that serve the whole group) and for launch waves of at most 64 MiB of
+ * activations (with 1 those take the sweeps too: their X is still in L2 at the next sweep);
+ * 0 = off: two sweeps over X per power step.  Default 1;
  * "wave_bytes" = activation bytes grouped into one launch wave of extraction;
  * "extract_streams" 2 (default) = alternate waves use two scratch regions and two helper
  * streams forked from and joined to the caller's stream, so that one wave's short kernels
@@ -208,7 +209,7 @@ agzo_status agzo_read_counters(agzo_ctx* ctx, double* h_ms, int64_t* h_timed_lau
  * the next call with the same array; its tables are uploaded on `stream`) and writes, per layer,
  * the thread-block cluster size with which its power steps run in the fused kernel, 0 for a
  * layer served by the two-sweep kernels (no X, the "extract_fused" / "extract_path" options,
- * its shape, or an X shared with a neighbouring layer).  h_cluster: host, n entries.  Launches
+ * its shape, an X shared with a neighbouring layer, or a launch wave small enough for L2).  h_cluster: host, n entries.  Launches
  * no kernel.                                                                               */
 agzo_status agzo_query_fused(agzo_ctx* ctx, const agzo_layer* h_layers, int n, int32_t* h_cluster,
                              void* stream);

@@ -18,6 +18,7 @@ constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;          // DevStatus + scalar slots
 constexpr size_t kCoefOffset = 64;            // float coefficient slot inside the header
 constexpr int64_t kDefaultWaveBytes = 8ll << 30;
+constexpr int64_t kL2ResidentWaveBytes = 64ll << 20;   // a wave's X up to this size is still in L2 at its next sweep
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
@@ -26,6 +27,7 @@ struct Plan {
   std::vector<int> tile_start;     // n + 1
   std::vector<int> wave_end;       // exclusive end index of each extraction wave
   std::vector<int> wave_region;    // scratch region (= helper stream) of each wave, -1 = nothing to do
+  std::vector<int64_t> wave_xbytes;   // activation bytes of each wave (a shared X counted once)
   // the Y panels of a wave's layers lie one after another at the end of the wave's scratch, so that a
   // token-sharded run can sum all of them over the ranks in one call
   std::vector<float*> wave_y;
@@ -242,6 +244,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   plan->tile_start.assign(n + 1, 0);
   plan->wave_end.clear();
   plan->wave_region.clear();
+  plan->wave_xbytes.clear();
   plan->wave_y.clear();
   plan->wave_y_count.clear();
   const int regions = opts.extract_regions == 2 ? 2 : 1;
@@ -358,7 +361,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   while (i < n) {
     if (!has_x(L[i])) {
       ++i;
-      plan->wave_end.push_back(i); plan->wave_region.push_back(-1);
+      plan->wave_end.push_back(i); plan->wave_region.push_back(-1); plan->wave_xbytes.push_back(0);
       plan->wave_y.push_back(nullptr); plan->wave_y_count.push_back(0);
       continue;
     }
@@ -454,10 +457,17 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       std::stable_sort(ord.begin(), ord.end(), [&](int a, int b) { return L[i + a].d_in > L[i + b].d_in; });
       for (int k = 0; k < j - i; ++k) plan->dev[i + k].xq_order = ord[k];
     }
-    if (ws)   // the fused kernel's launches of this wave, one per cluster size: who works on which tiles
+    if (ws) {
+      // A wave whose activations stay in L2 from one sweep to the next gains nothing from the fused kernel
+      // (its point is that X crosses HBM once per power step): such a wave takes the two sweeps throughout.
+      if (opts.extract_fused != 2 && xbytes <= kL2ResidentWaveBytes)
+        for (int k = i; k < j; ++k) plan->dev[k].fz_C = 0;
+      // the fused kernel's launches of this wave, one per cluster size: who works on which tiles
       for (int C = 1; C <= 16; ++C) fused_plan_shares(plan->dev.data(), i, j, C);
+    }
     plan->wave_end.push_back(j);
     plan->wave_region.push_back(region);
+    plan->wave_xbytes.push_back(xbytes);
     i = j;
   }
   if (scratch_needed) {

@@ -399,6 +399,44 @@ def test_extract_many_layers_in_waves():
             assert projector_distance(to_host(devs[i][1]), Vo) <= 1e-3
 
 
+def test_which_layers_take_the_fused_power_step():
+    """The default: a layer whose X is larger than an L2-sized wave and whose cluster size keeps most SMs busy
+    runs its power steps in the fused kernel; small waves, shared inputs and the option 0 do not."""
+    big = WL.planted_activations(9000, 4096, 16, seed=3, bf16=True)      # 74 MB of bf16
+    small = WL.planted_activations(512, 1024, 16, seed=4, bf16=True)
+    Xb, _ = to_dev(big, True)
+    Xs, _ = to_dev(small, True)
+    Vb = torch.zeros(8, 4096, device=DEV)
+    Vs = torch.zeros(8, 1024, device=DEV)
+    Vs2 = torch.zeros(8, 1024, device=DEV)
+    layers = [B.make_layer(X=Xb, V=Vb, r=8, layer_id=0), B.make_layer(X=Xs, V=Vs, r=8, layer_id=1)]
+    with Ctx(layers) as ctx:
+        cap = B.agzo_query_cluster_capacity(ctx)
+        sms = torch.cuda.get_device_properties(DEV).multi_processor_count
+        assert cap[0] == 0 and cap[1] == sms
+        assert all(cap[c] * c <= sms for c in range(1, 17))
+        assert all(cap[c] >= cap[c + 1] for c in range(1, 16))
+        B.agzo_set_option(ctx, "wave_bytes", 1)                 # one layer per wave
+        fz = B.agzo_query_fused(ctx, layers)
+        assert fz[1] == 0                                       # 1 MB of activations: stays in L2
+        assert fz[0] == (8 if cap[8] * 8 * 10 >= sms * 7 else 0)
+        B.agzo_extract_subspace(ctx, layers, 9, 3)
+        assert B.agzo_poll(ctx) == B.AGZO_OK
+        Vo = O.extract_subspace(big, 8, 3, 9, 0)
+        assert projector_distance(to_host(Vb), Vo) <= 1e-3
+        B.agzo_set_option(ctx, "extract_fused", 2)
+        assert B.agzo_query_fused(ctx, layers) == [8, 2]
+        B.agzo_set_option(ctx, "extract_fused", 0)
+        assert B.agzo_query_fused(ctx, layers) == [0, 0]
+    # two layers on one X: one sweep serves both, which beats one fused pass each
+    shared = [B.make_layer(X=Xs, V=Vs, r=8, layer_id=1), B.make_layer(X=Xs, V=Vs2, r=8, layer_id=2)]
+    with Ctx(shared) as ctx:
+        B.agzo_set_option(ctx, "wave_bytes", 1 << 40)
+        assert B.agzo_query_fused(ctx, shared) == [0, 0]
+        B.agzo_set_option(ctx, "extract_fused", 2)
+        assert B.agzo_query_fused(ctx, shared) == [2, 2]
+
+
 def test_extract_wave_mixes_fused_and_unfused_layers():
     # d_in = 4608 and r = 24 are beyond the fused kernel's shapes; the others run fused on clusters of 2, 1 and 4
     specs = [(640, 1024, 8), (512, 4608, 4), (700, 264, 16), (512, 512, 24), (768, 2048, 2)]
