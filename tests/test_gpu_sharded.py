@@ -66,8 +66,9 @@ def run_ranks(world, body):
     return results
 
 
-@pytest.mark.parametrize("path,K", [(1, 3), (2, 3), (2, 0)])
-def test_two_token_shards_give_the_whole_batch_subspace(path, K):
+@pytest.mark.parametrize("path,K,fused", [(1, 3, 0), (2, 3, 0), (2, 0, 0), (2, 3, 2)])
+def test_two_token_shards_give_the_whole_batch_subspace(path, K, fused):
+    # fused = 2: the power steps run in the cluster kernel, whose partial sums per layer are counted differently
     # the split points are odd, so a rank's first element of Omega falls inside a Philox block
     specs = [(1100, 256, 3, 517), (1536, 512, 8, 768), (900, 384, 6, 333)]   # m, d_in, r, tokens of rank 0
     seed = 21
@@ -90,6 +91,7 @@ def test_two_token_shards_give_the_whole_batch_subspace(path, K):
         for i, (m, d, r, m0) in enumerate(specs):          # one call per layer: the offsets differ
             with Ctx([layers[i]]) as ctx:
                 B.agzo_set_option(ctx, "extract_path", path)
+                B.agzo_set_option(ctx, "extract_fused", fused)
                 B.agzo_set_allreduce(ctx, hub.fn(rank), 0 if rank == 0 else m0)
                 B.agzo_extract_subspace(ctx, [layers[i]], seed, K, stream=stream)
                 stream.synchronize()
