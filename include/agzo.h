@@ -343,6 +343,18 @@ agzo_status agzo_debug_philox(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, u
 agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id, uint32_t tag,
                                 uint64_t first, uint64_t n, float* d_vals, void* stream);
 
+/* Test export, host only (no context, no device): the fused power step's work split.  Layer i has
+ * h_tiles[i] token tiles; the tiles of the n layers form one list that is cut into
+ * *h_shares = min(total, clusters) contiguous shares whose sizes differ by at most one tile.
+ * Outputs, all host: h_tile0[i] the layer's first tile in the list, h_first[i] the first share
+ * that meets the layer, h_parts[i] how many shares meet it (= its partial sums of Y after a power
+ * step; 0 for a layer without tiles), h_share_begin[0 .. *h_shares] the first tile of every share
+ * and the total (clusters + 1 entries of room).  AGZO_ERR_INVALID_ARG for clusters < 1, a negative
+ * count or more than 2^30 tiles.                                                            */
+agzo_status agzo_debug_fused_split(const int32_t* h_tiles, int n, int clusters, int32_t* h_tile0,
+                                   int32_t* h_first, int32_t* h_parts, int32_t* h_share_begin,
+                                   int32_t* h_shares);
+
 /* Exercises the bounded device-side wait that every pipeline of the tensor-core kernels uses:
  * launches one small block that waits, with the library's own wait routine, on a barrier that
  * nothing ever completes.  The wait gives up after its time limit (two seconds), the block

@@ -32,7 +32,7 @@ EXPORTS = [
     "agzo_restore", "agzo_update", "agzo_ghat", "agzo_restore_update", "agzo_step",
     "agzo_perturb_dense", "agzo_debug_philox", "agzo_debug_gaussian", "agzo_read_counters",
     "agzo_extract_subspace_static", "agzo_fill_gaussian_basis", "agzo_set_allreduce",
-    "agzo_debug_wait_timeout", "agzo_query_fused", "agzo_query_cluster_capacity",
+    "agzo_debug_wait_timeout", "agzo_query_fused", "agzo_query_cluster_capacity", "agzo_debug_fused_split",
 ]
 KC_RMW, KC_XT_T, KC_X_Q, KC_PANEL_QR, KC_TC_XT_T, KC_TC_X_Q, KC_OMEGA, KC_RMW_TC, KC_FUSED_POWER = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
@@ -103,6 +103,8 @@ def lib() -> C.CDLL:
         "agzo_debug_wait_timeout": (i32, [vp, vp]),
         "agzo_query_fused": (i32, [vp, LP, i32, C.POINTER(C.c_int32), vp]),
         "agzo_query_cluster_capacity": (i32, [vp, C.POINTER(C.c_int32)]),
+        "agzo_debug_fused_split": (i32, [C.POINTER(C.c_int32), i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                         C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
         "agzo_extract_subspace_static": (i32, [vp, i64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                C.c_int32, u64, u32, vp, i64, vp, vp]),
     }
@@ -231,6 +233,18 @@ def agzo_query_fused(ctx: Context, layers, stream=None, arr=None):
     out = (C.c_int32 * len(layers))()
     _check(lib().agzo_query_fused(ctx.handle, arr, len(layers), out, _stream_ptr(stream)), "agzo_query_fused")
     return list(out)
+
+
+def agzo_debug_fused_split(tiles, clusters: int):
+    """(tile0, first, parts, share_begin) of the fused power step's work split; host arithmetic only."""
+    n = len(tiles)
+    t = (C.c_int32 * max(n, 1))(*tiles)
+    tile0, first, parts = (C.c_int32 * max(n, 1))(), (C.c_int32 * max(n, 1))(), (C.c_int32 * max(n, 1))()
+    begin = (C.c_int32 * (clusters + 1))()
+    shares = C.c_int32(0)
+    _check(lib().agzo_debug_fused_split(t, n, clusters, tile0, first, parts, begin, C.byref(shares)),
+           "agzo_debug_fused_split")
+    return list(tile0)[:n], list(first)[:n], list(parts)[:n], list(begin)[:shares.value + 1]
 
 
 def agzo_query_cluster_capacity(ctx: Context):

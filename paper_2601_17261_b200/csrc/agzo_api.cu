@@ -1112,6 +1112,23 @@ agzo_status agzo_debug_gaussian(agzo_ctx* ctx, uint64_t seed, uint32_t layer_id,
   return AGZO_OK;
 }
 
+agzo_status agzo_debug_fused_split(const int32_t* h_tiles, int n, int clusters, int32_t* h_tile0, int32_t* h_first,
+                                   int32_t* h_parts, int32_t* h_share_begin, int32_t* h_shares) {
+  if (n < 0 || clusters < 1 || (n > 0 && (!h_tiles || !h_tile0 || !h_first || !h_parts)) || !h_share_begin || !h_shares)
+    return AGZO_ERR_INVALID_ARG;
+  long long total = 0;
+  for (int i = 0; i < n; ++i) {
+    if (h_tiles[i] < 0) return AGZO_ERR_INVALID_ARG;
+    total += h_tiles[i];
+  }
+  if (total > (1ll << 30)) return AGZO_ERR_INVALID_ARG;
+  int base = 0, rem = 0;
+  const int G = fused_split(h_tiles, n, clusters, h_tile0, h_first, h_parts, &base, &rem);
+  for (int k = 0; k <= G; ++k) h_share_begin[k] = fused_share_begin(k, base, rem);
+  *h_shares = G;
+  return AGZO_OK;
+}
+
 agzo_status agzo_debug_wait_timeout(agzo_ctx* ctx, void* stream) {
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;

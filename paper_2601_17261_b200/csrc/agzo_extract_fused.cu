@@ -32,6 +32,8 @@
 // status word and the CTA leaves through the common exit (cluster barrier, TMEM freed).
 #include <cuda.h>
 
+#include <vector>
+
 #include "agzo_ptx.cuh"
 #include "agzo_tc.cuh"
 
@@ -579,26 +581,46 @@ int fused_parts_bound(const agzo_layer& a, int C) {
   return nt < shares ? nt : shares;
 }
 
-// Cuts the tiles of the layers of [l0, l1) with cluster size C into shares: fills fz_tile0 and fz_parts.
-void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
+// The arithmetic of the work split on plain arrays (also what the host-side test export runs): layer i has
+// tiles[i] tiles; with `clusters` resident clusters there are G = min(total, clusters) shares.  Writes each
+// layer's first tile in the list, the first share that meets it and the number of shares that do; returns G
+// and the share sizes (base, rem: the first rem shares have base + 1 tiles).
+int fused_split(const int* tiles, int n, int clusters, int* tile0, int* first, int* parts, int* base, int* rem) {
   int total = 0;
+  for (int i = 0; i < n; ++i) { tile0[i] = total; total += tiles[i]; }
+  if (total == 0) { *base = 0; *rem = 0; return 0; }
+  const int cap = clusters > 0 ? clusters : 1;
+  const int G = total < cap ? total : cap;
+  *base = total / G;
+  *rem = total % G;
+  for (int i = 0; i < n; ++i) {
+    first[i] = fz_share_of(tile0[i], *base, *rem);
+    parts[i] = tiles[i] > 0 ? fz_share_of(tile0[i] + tiles[i] - 1, *base, *rem) - first[i] + 1 : 0;
+  }
+  return G;
+}
+int fused_share_begin(int k, int base, int rem) { return fz_share_begin(k, base, rem); }
+
+// Cuts the tiles of the layers of [l0, l1) with cluster size C into shares: fills fz_tile0, fz_first and fz_parts.
+void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
+  std::vector<int> idx, tiles;
   bool wide = C > 8;
   for (int i = l0; i < l1; ++i)
     if (dev[i].fz_C == C) {
-      dev[i].fz_tile0 = total;
-      total += (dev[i].m + kTT - 1) / kTT;
+      idx.push_back(i);
+      tiles.push_back((dev[i].m + kTT - 1) / kTT);
       wide = wide || dev[i].fz_slice > kSliceCols;
     }
-  if (total == 0) return;
-  const int cap = g_max_clusters[wide][C] > 0 ? g_max_clusters[wide][C] : 1;
-  const int G = total < cap ? total : cap;
-  const int base = total / G, rem = total % G;
-  for (int i = l0; i < l1; ++i)
-    if (dev[i].fz_C == C) {
-      const int nt = (dev[i].m + kTT - 1) / kTT;
-      dev[i].fz_first = fz_share_of(dev[i].fz_tile0, base, rem);
-      dev[i].fz_parts = fz_share_of(dev[i].fz_tile0 + nt - 1, base, rem) - dev[i].fz_first + 1;
-    }
+  if (idx.empty()) return;
+  const int n = (int)idx.size();
+  std::vector<int> tile0(n), first(n), parts(n);
+  int base = 0, rem = 0;
+  fused_split(tiles.data(), n, g_max_clusters[wide][C], tile0.data(), first.data(), parts.data(), &base, &rem);
+  for (int k = 0; k < n; ++k) {
+    dev[idx[k]].fz_tile0 = tile0[k];
+    dev[idx[k]].fz_first = first[k];
+    dev[idx[k]].fz_parts = parts[k];
+  }
 }
 
 // One fused power step for the layers of the wave whose cluster size is C.

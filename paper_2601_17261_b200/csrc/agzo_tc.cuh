@@ -62,6 +62,9 @@ int fused_slice_cols(const agzo_layer& a, bool any_size);   // columns of X per 
 int fused_parts_bound(const agzo_layer& a, int C);              // partial sums of Y a power step can leave, at most
 void fused_plan_shares(DevLayer* dev, int l0, int l1, int C);   // fills fz_tile0 / fz_parts of a wave's layers of size C
 int fused_resident_clusters(int C);                             // clusters of C CTAs the device holds at once (after fused_init)
+// the split on plain arrays and the first tile of share k (host; the kernel walks the same shares)
+int fused_split(const int* tiles, int n, int clusters, int* tile0, int* first, int* parts, int* base, int* rem);
+int fused_share_begin(int k, int base, int rem);
 cudaError_t fused_init(int sm_count);          // asks the device which cluster sizes fit; eligibility follows it
 cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
                                     cudaStream_t s);

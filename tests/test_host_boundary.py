@@ -94,6 +94,46 @@ def test_calls_on_a_null_context_fail_cleanly(lib):
     assert lib.agzo_set_allreduce(None, B.ALLREDUCE_FN(), None, 0) == B.AGZO_ERR_STATE
 
 
+def test_fused_work_split_covers_every_tile_once(lib):
+    """The fused power step cuts the tiles of a launch's layers into one contiguous share per cluster.
+    Whatever the layer sizes: every tile belongs to exactly one share, the shares differ by at most one
+    tile, and a layer's partial sums are numbered 0 .. parts - 1 without gaps, one per share that meets it."""
+    import random
+    rng = random.Random(7)
+    cases = [([128] * 24, 15), ([128] * 6 + [128], 16), ([64] * 168, 74), ([1], 148), ([5, 0, 3], 2), ([7], 3)]
+    for _ in range(300):
+        cases.append(([rng.randint(1, 140) for _ in range(rng.randint(1, 50))], rng.randint(1, 148)))
+    for tiles, clusters in cases:
+        tile0, first, parts, begin = B.agzo_debug_fused_split(tiles, clusters)
+        total = sum(tiles)
+        G = len(begin) - 1
+        assert G == min(total, clusters)
+        assert begin[0] == 0 and begin[-1] == total
+        sizes = [begin[k + 1] - begin[k] for k in range(G)]
+        assert min(sizes) >= 1 and max(sizes) - min(sizes) <= 1
+        assert tile0 == [sum(tiles[:i]) for i in range(len(tiles))]
+        covered = [[0] * t for t in tiles]
+        seen = [set() for _ in tiles]
+        for k in range(G):                                   # what cluster k does, as the kernel walks it
+            for i, t in enumerate(tiles):
+                b, e = max(begin[k], tile0[i]), min(begin[k + 1], tile0[i] + t)
+                if b >= e:
+                    continue
+                part = k - first[i]
+                assert 0 <= part < parts[i] and part not in seen[i]
+                seen[i].add(part)
+                for x in range(b - tile0[i], e - tile0[i]):
+                    covered[i][x] += 1
+        assert all(c == 1 for cv in covered for c in cv)
+        assert [len(sv) for sv in seen] == parts
+        assert all(p <= min(t, G) for p, t in zip(parts, tiles))
+    bad = (C.c_int32 * 1)(-1)
+    out = (C.c_int32 * 4)()
+    n = C.c_int32(0)
+    assert lib.agzo_debug_fused_split(bad, 1, 4, out, out, out, out, C.byref(n)) == B.AGZO_ERR_INVALID_ARG
+    assert lib.agzo_debug_fused_split(bad, 1, 0, out, out, out, out, C.byref(n)) == B.AGZO_ERR_INVALID_ARG
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libagzo.so")
