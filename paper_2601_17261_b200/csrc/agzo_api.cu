@@ -81,7 +81,7 @@ struct agzo_ctx {
   int rmw_stage_r;         // 0 auto, 1 never, 2 always
   int64_t wave_bytes;
   int extract_streams;     // 1 or 2 (see PlanOpts::extract_regions)
-  int extract_fused;       // 1: fused power-step kernel where a layer's shape allows it
+  int extract_fused;       // 0 off, 1 fused power-step kernel where it pays, 2 wherever a layer's shape allows it
   int share_inputs;        // 1: consecutive layers with the same X share the sweeps over it
   // staged R images in scratch: valid for this seed until the plan changes or extraction uses the scratch
   bool rimg_valid;
@@ -617,7 +617,7 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, 0, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
-  // ... and for the fused power step, whose layers keep short token slabs
+  // ... and for the fused power step, whose layers keep room for one partial sum of Y per share of a launch
   st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 2, false, 2}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;

@@ -52,17 +52,33 @@ constexpr int kWideSliceCols = 768;        // ... and where 16 such slices do no
 constexpr int kMaxCluster = 16;
 constexpr int kSlotBytes = 16 * 1024;      // ring A: [128 tokens][64 columns]; ring C: [64 tokens][128 columns]
 constexpr int kBoxBytes = 8 * 1024;        // one TMA box of 64 tokens x 64 columns
-constexpr int kRingC = 4;                  // ring A: 5 slots, 4 beside the Q region of a wide slice
-constexpr int kMaxRing = 8;
+constexpr int kMaxRingSlots = 8;
 constexpr int kLook = 2;                   // phase A runs up to this many tiles ahead of phase C
 constexpr int kBuf = kLook + 1;            // T partial (TMEM) and T operand (shared memory) buffers in rotation
 constexpr int kRs = 2;                     // exchange buffers in rotation
-constexpr int kRsFloats = 2688;            // C * ceil(16 / C) * 8 * NP floats at most (C = 7, NP = 16)
-constexpr int kTtBytes = 32 * 256;         // T operand: up to 32 rows of 128 tokens
+
+// Shared-memory budget of an instantiation.  kWide: 768-column slices (12 boxes of Q instead of 8) or clusters
+// of more than 8 CTAs.  kSmall: every layer of the launch has r <= 8, i.e. NB <= 16 operand rows: the Q slice,
+// the T operands and the exchange buffers are half as large and the rings get the room (the kernel's rate
+// follows the bytes its rings keep in flight).
+template <bool kWide, bool kSmall>
+struct FzCfg {
+  static constexpr int nb_max = kSmall ? 16 : 32;
+  static constexpr int q_bytes = (kWide ? 12 : 8) * nb_max * 128;
+  static constexpr int tt_bytes = nb_max * 256;                 // T operand: nb_max rows of 128 tokens
+  // exchange buffer: C * ceil(16 / C) * 8 * NP floats at most (NP = 16: C = 7; NP = 8: C = 15)
+  static constexpr int rs_floats = kSmall ? 1920 : 2688;
+  static constexpr int ring_a = kSmall ? (kWide ? 5 : 6) : (kWide ? 4 : 5);
+  static constexpr int ring_c = kSmall ? 5 : 4;
+  static constexpr size_t smem = (size_t)(ring_a + ring_c) * kSlotBytes + q_bytes + kBuf * tt_bytes +
+                                 kRs * rs_floats * 4 + 8 * 512 + 1024;
+  static_assert(ring_a <= kMaxRingSlots && ring_c <= kMaxRingSlots, "barrier arrays");
+  static_assert(smem + 1024 <= 227 * 1024, "shared memory per CTA");
+};
 
 struct FzShared {
-  uint64_t xa_full[kMaxRing], xa_empty[kMaxRing];
-  uint64_t xc_full[kMaxRing], xc_empty[kMaxRing];
+  uint64_t xa_full[kMaxRingSlots], xa_empty[kMaxRingSlots];
+  uint64_t xc_full[kMaxRingSlots], xc_empty[kMaxRingSlots];
   uint64_t qb_full, qb_empty;
   uint64_t tp_full[kBuf], tp_empty[kBuf];     // T partial in TMEM
   uint64_t tt_full[kBuf];                     // T operand in shared memory: the owners' sums have landed
@@ -117,9 +133,8 @@ __device__ __forceinline__ uint32_t swz(int i, int j) {
 
 // kWide: some layer of the launch has 768-column slices (its Q slice takes 12 boxes instead of 8, so ring A
 // has one slot less, and its six Y accumulators need more than 256 TMEM columns) or the cluster has more
-// than 8 CTAs.  Two instantiations, because only the wide one is marked for cluster sizes beyond the
-// portable 8.
-template <bool kWide>
+// than 8 CTAs; only the wide instantiations are marked for cluster sizes beyond the portable 8.
+template <bool kWide, bool kSmall>
 __global__ void __launch_bounds__(kFzThreads, 1)
 fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int C, int share_base, int share_rem,
                         DevStatus* status) {
@@ -129,14 +144,16 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();
   const int cluster = (int)cluster_id_x();
-  constexpr int ring_a = kWide ? 4 : 5;
+  using Cfg = FzCfg<kWide, kSmall>;
+  constexpr int ring_a = Cfg::ring_a, kRingC = Cfg::ring_c;
+  constexpr int kTtBytes = Cfg::tt_bytes, kRsFloats = Cfg::rs_floats;
   constexpr uint32_t tmem_cols = kWide ? 512u : 256u;
   // shared-memory carve-up: ring A | ring C | Q slice (boxes of [NB][64]) | T operand x kBuf | exchange buffers x kRs | staging
   uint8_t* sXA = base;
   uint8_t* sXC = sXA + (size_t)ring_a * kSlotBytes;
   uint8_t* sQ = sXC + (size_t)kRingC * kSlotBytes;
-  // NB is a per-layer quantity; the regions are sized for NB = 32
-  uint8_t* sTt = sQ + (kWide ? 12 : 8) * 32 * 128;
+  // NB is a per-layer quantity; the regions are sized for the instantiation's largest NB
+  uint8_t* sTt = sQ + Cfg::q_bytes;
   float* sRs = reinterpret_cast<float*>(sTt + kBuf * kTtBytes);   // kRs x [C][cpo][8][NP] floats
   uint8_t* sStage = reinterpret_cast<uint8_t*>(sRs + kRs * kRsFloats);   // 512 bytes per epilogue warp
 
@@ -489,8 +506,14 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
 int g_max_clusters[2][kMaxCluster + 1] = {};   // [narrow / wide instantiation][cluster size]
 int g_sm_count = 0;                         // 0 until fused_init has run
 
-size_t fz_smem_bytes() {
-  return (size_t)(5 + kRingC) * kSlotBytes + 8 * 32 * 128 + kBuf * kTtBytes + kRs * kRsFloats * 4 + 8 * 512 + 1024;
+using FzKernel = void (*)(const DevLayer*, int, int, int, int, int, DevStatus*);
+FzKernel fz_kernel(bool wide, bool small) {
+  return wide ? (small ? fused_power_step_kernel<true, true> : fused_power_step_kernel<true, false>)
+              : (small ? fused_power_step_kernel<false, true> : fused_power_step_kernel<false, false>);
+}
+size_t fz_smem_bytes(bool wide, bool small) {
+  return wide ? (small ? FzCfg<true, true>::smem : FzCfg<true, false>::smem)
+              : (small ? FzCfg<false, true>::smem : FzCfg<false, false>::smem);
 }
 
 cudaError_t fz_max_clusters(bool wide, int C, int sm_count, int* n) {
@@ -502,11 +525,10 @@ cudaError_t fz_max_clusters(bool wide, int C, int sm_count, int* n) {
   attr[0].val.clusterDim.z = 1;
   cfg.blockDim = dim3(kFzThreads);
   cfg.gridDim = dim3((unsigned)(C * (sm_count / C)));
-  cfg.dynamicSmemBytes = fz_smem_bytes();
+  cfg.dynamicSmemBytes = fz_smem_bytes(wide, false);     // one CTA per SM in every instantiation
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return wide ? cudaOccupancyMaxActiveClusters(n, fused_power_step_kernel<true>, &cfg)
-              : cudaOccupancyMaxActiveClusters(n, fused_power_step_kernel<false>, &cfg);
+  return cudaOccupancyMaxActiveClusters(n, (const void*)fz_kernel(wide, false), &cfg);
 }
 
 }  // namespace
@@ -527,7 +549,8 @@ int fused_slice_cols(const agzo_layer& a, bool any_size) {
   for (int slice : {kSliceCols, kWideSliceCols}) {
     const int C = (a.d_in + slice - 1) / slice;
     if (C > kMaxCluster) continue;
-    if (C * ((kGroups + C - 1) / C) * 8 * NP > kRsFloats) continue;
+    if (C * ((kGroups + C - 1) / C) * 8 * NP > (NP <= 8 ? FzCfg<false, true>::rs_floats : FzCfg<false, false>::rs_floats))
+      continue;
     double share = 0.0;
     if (g_sm_count) {
       const int resident = g_max_clusters[slice > kSliceCols || C > 8][C];
@@ -550,15 +573,17 @@ bool fused_eligible(const agzo_layer& a, bool any_size) {
 }
 
 cudaError_t fused_init(int sm_count) {
-  cudaError_t e = cudaFuncSetAttribute(fused_power_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)fz_smem_bytes());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(fused_power_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)fz_smem_bytes());
-  if (e != cudaSuccess) return e;
-  // clusters of more than 8 CTAs are beyond the portable size: ask for them, and use them only if they fit
-  const bool big = cudaFuncSetAttribute(fused_power_step_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed,
-                                        1) == cudaSuccess;
+  bool big = true;
+  for (int wide = 0; wide < 2; ++wide)
+    for (int small = 0; small < 2; ++small) {
+      cudaError_t e = cudaFuncSetAttribute((const void*)fz_kernel(wide, small), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)fz_smem_bytes(wide, small));
+      if (e != cudaSuccess) return e;
+      // clusters of more than 8 CTAs are beyond the portable size: ask for them, and use them only if they fit
+      if (wide && cudaFuncSetAttribute((const void*)fz_kernel(true, small), cudaFuncAttributeNonPortableClusterSizeAllowed,
+                                       1) != cudaSuccess)
+        big = false;
+    }
   for (int C = 1; C <= kMaxCluster; ++C) {
     int n = 0;
     if (C > 8 || fz_max_clusters(false, C, sm_count, &n) != cudaSuccess) n = 0;
@@ -627,11 +652,12 @@ void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
 cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
                                     cudaStream_t s) {
   int total = 0;
-  bool wide = C > 8;
+  bool wide = C > 8, small = true;
   for (int i = w.l0; i < w.l1; ++i)
     if (h_dev[i].fz_C == C) {
       total += (h_dev[i].m + kTT - 1) / kTT;
       if (h_dev[i].fz_slice > kSliceCols) wide = true;
+      if (h_dev[i].NB > 16) small = false;
     }
   if (total == 0) return cudaSuccess;
   if (C < 1 || C > kMaxCluster || g_max_clusters[wide][C] <= 0) return cudaErrorInvalidConfiguration;   // the planner picks no such size
@@ -642,7 +668,7 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.blockDim = dim3(kFzThreads);
-  cfg.dynamicSmemBytes = fz_smem_bytes();
+  cfg.dynamicSmemBytes = fz_smem_bytes(wide, small);
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
@@ -653,8 +679,7 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   int l0 = w.l0, l1 = w.l1;
   int base = total / nclusters, rem = total % nclusters;
   void* args[] = {(void*)&layers, (void*)&l0, (void*)&l1, (void*)&C, (void*)&base, (void*)&rem, (void*)&d_status};
-  return wide ? cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel<true>, args)
-                         : cudaLaunchKernelExC(&cfg, (const void*)fused_power_step_kernel<false>, args);
+  return cudaLaunchKernelExC(&cfg, (const void*)fz_kernel(wide, small), args);
 }
 
 }  // namespace agzo
