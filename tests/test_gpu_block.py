@@ -191,6 +191,9 @@ def test_extraction_inside_the_forward_of_an_8b_shaped_block():
         g = torch.Generator(device="cpu").manual_seed(5)
         x0 = torch.randn(batch, seq, 4096, generator=g).to(DEV).to(torch.bfloat16)
         with torch.no_grad():
+            blk(x0)                       # first pass: the kernels' modules are loaded, the library has planned once
+            torch.cuda.synchronize()
+            events.clear()
             out = blk(x0)
         torch.cuda.synchronize()
         assert B.agzo_poll(ctx) == B.AGZO_OK
