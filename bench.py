@@ -35,7 +35,7 @@ K_POWER = 3
 # slice of the 8B-shaped layer set (summaries under profiles/); traffic grows in proportion
 # to the activation bytes a launch sweeps.  Reset an entry to None when its kernel changes.
 TRAFFIC_PER_ALGORITHMIC_BYTE = {"tc_xt_t_kernel": (4.865880 + 0.011429) / 4.831838,
-                                "fused_power_step_kernel": (3.272740 + 0.009301) / 3.221225}
+                                "fused_power_step_kernel": (3.272938 + 0.009340) / 3.221225}
 # Thread-level instructions per weight of the dense-direction kernel (one Philox + Box-Muller normal per weight):
 # ncu smsp__thread_inst_executed.sum / weights on a 4096 x 4096 bf16 layer (profiles/dense_vec_kernel_*.md).
 DENSE_INST_PER_WEIGHT = 933126144 / (4096 * 4096)
