@@ -3,7 +3,7 @@
 // The two products of a power step meet the same X: T = X Q needs a whole row of X (all of d_in)
 // before a single element of Y = X^T T can be formed, so the unfused kernels read X twice from
 // HBM.  Here a thread-block cluster of C CTAs shares a tile of 128 tokens; CTA c works on its
-// slice of the tile's columns (512 of them in clusters of up to 16; 768 where d_in is beyond 16 x 512):
+// slice of the tile's columns (512 or 768 of them, whichever keeps more of the device busy; C <= 16):
 //   phase A   the slice's contribution to T (128 x NB, tcgen05.mma M = 128) goes to TMEM;
 //             X streams through a ring of shared-memory slots (first read, from HBM, marked
 //             evict-last for L2) and every slot is released as soon as its MMAs have read it,
@@ -11,10 +11,11 @@
 //             hops (st.async): groups of eight token rows are summed in rank order by the CTA that
 //             owns them, which writes the bf16 hi/lo parts of the sums straight into the T operand
 //             buffer of every CTA of the cluster,
-//   phase C   Y_slice (slice x NB, kept in TMEM across all tiles of the work item) += X_slice^T T;
-//             the slice is fetched a second time through a second, smaller ring -- a few boxes
-//             behind the first read, so it comes from L2 (measured: a line survives 20 to 50 MB of
-//             streaming traffic, and this lag is about one tile per CTA).
+//   phase C   Y_slice (slice x NB, kept in TMEM across a whole run of tiles) += X_slice^T T;
+//             the slice is fetched a second time through a second ring with its own producer,
+//             two to three tiles behind the first read, so it comes from L2 (measured: a line
+//             survives 20 to 50 MB of streaming traffic; this lag is 33 to 50 MB over the grid,
+//             and the DRAM counters show X crossing once).
 // An earlier version kept the tile resident in shared memory between the phases; the exchange
 // takes about 2 us, the ring held 2.5 tiles of 64 KiB, and that residency, not the arithmetic,
 // bounded it at 3.6 TB/s.  The tiles of all layers of a launch form one list that is cut into equal
@@ -24,12 +25,17 @@
 // As in the unfused kernels Q and T are fp32 quantities carried as hi + lo bf16 pairs in NB = 2 NP
 // operand columns (NP = r rounded up to 8), products exact, accumulation fp32.
 //
-// Roles in a CTA: warp 0 TMA producer of ring A (and of the Q slice, once per item), warp 10 TMA
-// producer of ring C, warp 1 MMA issuer (all lanes run the loop, an elected lane issues; phase A of
-// tile i+1 is issued before phase C of tile i so that the exchange of one tile overlaps the loads
-// and phase A of the next), two groups of four epilogue warps that take alternate tiles (TMEM ->
-// exchange; group 0 also writes Y out).  Every wait is bounded; a wait that runs out sets the
-// status word and the CTA leaves through the common exit (cluster barrier, TMEM freed).
+// Roles in a CTA: warp 0 TMA producer of ring A (and of the Q slice, once per piece of the share),
+// warp 10 TMA producer of ring C, warp 1 MMA issuer (all lanes run the loop, an elected lane issues;
+// it takes whichever phase has its operands, phase A up to two tiles ahead of phase C, so that the
+// exchange of a tile overlaps the loads and MMAs of the next two), two groups of four epilogue warps
+// that take alternate tiles (TMEM -> exchange; group 0 also writes Y out).  Every wait is bounded; a
+// wait that runs out sets the status word and the CTA leaves through the common exit (cluster
+// barrier, TMEM freed).
+//
+// The MMA warp's addresses and descriptors must stay values the compiler can prove warp-uniform (they
+// travel in uniform registers); a 64-bit division in this kernel once broke that proof for everything
+// after it and cost a third of the kernel's rate, which is why the share arithmetic is the host's.
 #include <cuda.h>
 
 #include <vector>
