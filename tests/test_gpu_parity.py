@@ -399,6 +399,33 @@ def test_extract_many_layers_in_waves():
             assert projector_distance(to_host(devs[i][1]), Vo) <= 1e-3
 
 
+def test_fused_shares_cross_layers_of_different_rank():
+    """Layers of one cluster size form one tile list that is cut into contiguous shares, so a cluster's share
+    runs from one layer into the next: ranks 3, 16 and 8 (8- and 16-column operand panels, the launch sized
+    for the largest), token counts that are no multiples of the tile, more tiles than clusters and fewer."""
+    for specs in ([(900, 1024, 3), (1500, 1024, 16), (700, 1024, 8), (300, 1024, 16)],
+                  [(20000, 512, 8), (9000, 512, 4)],          # one CTA per cluster: 227 tiles over up to 148 shares
+                  [(640, 2048, 16), (640, 2048, 5)]):
+        Xs = [WL.planted_activations(m, d, 16, seed=70 + i, bf16=True) for i, (m, d, r) in enumerate(specs)]
+        devs, layers = [], []
+        for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
+            Xd, _ = to_dev(X, True)
+            Vd = torch.zeros(r, d, device=DEV)
+            devs.append((Xd, Vd))
+            layers.append(B.make_layer(X=Xd, V=Vd, r=r, layer_id=i))
+        with Ctx(layers) as ctx:
+            B.agzo_set_option(ctx, "extract_fused", 2)
+            fz = B.agzo_query_fused(ctx, layers)
+            assert len(set(fz)) == 1 and fz[0] > 0, fz
+            B.agzo_extract_subspace(ctx, layers, 11, 2)
+            assert B.agzo_poll(ctx) == B.AGZO_OK
+        for i, ((m, d, r), X) in enumerate(zip(specs, Xs)):
+            Vo = O.extract_subspace(X, r, 2, 11, i)
+            Vg = to_host(devs[i][1])
+            assert projector_distance(Vg, Vo) <= 1e-3, (specs, i)
+            assert np.abs(Vg - Vo).max() <= 1e-3, (specs, i)
+
+
 def test_which_layers_take_the_fused_power_step():
     """The default: a layer whose X is larger than an L2-sized wave and whose cluster size keeps most SMs busy
     runs its power steps in the fused kernel; small waves, shared inputs and the option 0 do not."""
