@@ -157,126 +157,28 @@ cudaError_t launch_x_q(const ExtractWave& w, cudaStream_t s) {
 }
 
 // ------------------------------------------------------------------ qr(Y), stage 1
-// Y[k][d] = sum_s Ypart[s][k][d] (fixed order) and the partial Gram matrix of this block's
-// columns in double.  A block takes kGramGroup chunks of 128 columns one after another and keeps
-// its sums in registers across them: thread = (4 x 4 block of the Gram matrix, part of the
-// columns), so every pair of loaded values feeds 16 multiply-adds.
+// Y[k][d] = sum_s Ypart[s][k][d] (fixed order) and the partial Gram matrix of this block's columns in double.
+// A block takes kGramGroup chunks of 128 columns one after another and keeps its sums in registers across
+// them.  The panel is fetched four columns per load with a batch of independent loads per thread: the fetch
+// latency is what this kernel used to wait for.  The products run on the FP64 tensor cores (mma.sync m8n8k4,
+// true double multiply-adds; tcgen05 has no FP64 form): the Gram matrix is cut into 8 x 8 tiles, a warp owns
+// whole tiles of the upper triangle and runs through all columns of the block's chunks for them, so no sums
+// cross warps and the order of additions is fixed.  Fragments (PTX ISA, m8n8k4 .f64): lane l holds
+// A[l / 4][l % 4], B[l % 4][l / 4] and D[l / 4][2 (l % 4) + {0, 1}]; with A = Y[8 bi ..][c ..] and
+// B = Y[8 bj ..][c ..]^T both operands are the element (l / 4, l % 4) of a row block of the staged chunk.  Rows
+// of the chunk are 132 floats apart, so the 8 x 4 elements a warp reads fall into 32 different banks.
 constexpr int kGramCols = 128;
 constexpr int kGramGroup = 4;
-__host__ __device__ inline int gram_csplit(int r4) {   // column parts per chunk: as many as 256 threads allow
-  const int nsq = (r4 >> 2) * (r4 >> 2);
-  int cs = 16;
-  while (cs > 1 && cs * nsq > 256) cs >>= 1;
-  return cs;
-}
-__host__ __device__ inline size_t gram_smem_bytes(int r) {
-  const int r4 = (r + 3) & ~3;
-  const size_t y = (size_t)r4 * kGramCols * sizeof(float);
-  const size_t red = (size_t)gram_csplit(r4) * r4 * r4 * sizeof(double);
-  return y > red ? y : red;
-}
-// the launch serves layers of several ranks, and the need is not monotone in r (fewer column
-// parts fit at larger r): take the largest need over all ranks up to the wave's maximum
-inline size_t gram_smem_bytes_upto(int max_r) {
-  size_t b = 0;
-  for (int r = 1; r <= max_r; ++r) b = gram_smem_bytes(r) > b ? gram_smem_bytes(r) : b;
-  return b;
-}
-__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0, int y_reduced,
-                                                          int after_fused) {
-  const DevLayer& L = layers[l0 + blockIdx.y];
-  const int nparts = y_parts(L, after_fused);
-  const int ngroups = (L.gchunks + kGramGroup - 1) / kGramGroup;
-  const int grp = blockIdx.x;
-  if (grp >= ngroups) return;
-  extern __shared__ __align__(16) unsigned char gram_smem[];
-  float* sY = reinterpret_cast<float*>(gram_smem);        // [r4][kGramCols]; later reused for the column parts' sums
-  const int r = L.r, r4 = (r + 3) & ~3, nb = r4 >> 2;
-  const int csplit = gram_csplit(r4), clen = kGramCols / csplit;
-  const int unit = threadIdx.x;
-  const int sq = unit / csplit, cs = unit - sq * csplit;
-  const int bi = sq / nb, bj = sq - bi * nb;
-  const bool busy = sq < nb * nb && bj >= bi;               // upper triangle of 4 x 4 blocks
-  double acc[4][4];
-#pragma unroll
-  for (int a = 0; a < 4; ++a)
-#pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
-  const int rot = threadIdx.x & 31;
-  for (int sub = 0; sub < kGramGroup; ++sub) {
-    const int chunk = grp * kGramGroup + sub;
-    if (chunk >= L.gchunks) break;
-    const int d0 = chunk * kGramCols;
-    __syncthreads();                                        // the previous chunk's values have been used
-    for (int i = threadIdx.x; i < r4 * kGramCols; i += 256) {
-      const int k = i / kGramCols, c = i - k * kGramCols;
-      const int d = d0 + c;
-      float y = 0.f;
-      if (k < r && d < L.d_in) {
-        if (y_reduced) {
-          y = L.Y[(long long)k * L.d_in + d];
-        } else {
-          for (int s = 0; s < nparts; ++s) y += L.Ypart[((long long)s * r + k) * L.d_in + d];
-          L.Y[(long long)k * L.d_in + d] = y;
-        }
-      }
-      sY[i] = y;
-    }
-    __syncthreads();
-    if (busy) {
-      const float* yi = sY + (4 * bi) * kGramCols;
-      const float* yj = sY + (4 * bj) * kGramCols;
-      // rows are 128 floats apart, so all rows share a bank at equal c: every lane starts at its own
-      // column of its part (a fixed rotation, so the sum is the same on every run)
-      for (int c = 0; c < clen; ++c) {
-        const int cc = cs * clen + ((c + rot) & (clen - 1));
-        double a[4], b[4];
-#pragma unroll
-        for (int x = 0; x < 4; ++x) { a[x] = (double)yi[x * kGramCols + cc]; b[x] = (double)yj[x * kGramCols + cc]; }
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-#pragma unroll
-          for (int y = 0; y < 4; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
-      }
-    }
-  }
-  // the column parts of a block are added in a fixed order through shared memory
-  __syncthreads();
-  double* red = reinterpret_cast<double*>(gram_smem);     // [csplit][r4][r4]
-  if (busy) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x)
-#pragma unroll
-      for (int y = 0; y < 4; ++y) red[((size_t)cs * r4 + 4 * bi + x) * r4 + 4 * bj + y] = acc[x][y];
-  }
-  __syncthreads();
-  double* out = L.Gpart + (long long)grp * r * r;
-  for (int p = threadIdx.x; p < r * r; p += 256) {
-    const int i = p / r, j = p - i * r;
-    if (j < i) continue;
-    double t = 0.0;
-    for (int q = 0; q < csplit; ++q) t += red[((size_t)q * r4 + i) * r4 + j];
-    out[p] = t;
-  }
-}
-
-// The same reduction for larger ranks, on the FP64 tensor cores (mma.sync m8n8k4, true double multiply-adds;
-// tcgen05 has no FP64 form): the Gram matrix is cut into 8 x 8 tiles, a warp owns whole tiles of the upper
-// triangle and runs through all columns of the block's chunks for them, so no sums cross warps and the
-// order of additions is fixed.  Fragments (PTX ISA, m8n8k4 .f64): lane l holds A[l / 4][l % 4],
-// B[l % 4][l / 4] and D[l / 4][2 (l % 4) + {0, 1}]; with A = Y[8 bi ..][c ..] and B = Y[8 bj ..][c ..]^T both
-// operands are the element (l / 4, l % 4) of a row block of the staged chunk.  Rows of the chunk are 132
-// floats apart, so the 8 x 4 elements a warp reads fall into 32 different banks.
 constexpr int kGramPitch = kGramCols + 4;
-constexpr int kGramMmaMinRank = 16;            // waves whose largest rank exceeds this take the tensor-core form
+constexpr int kApplyMmaMinRank = 16;           // Q = Y M: waves whose largest rank exceeds this take the tensor-core form
 constexpr int kGramMmaTilesPerWarp = 5;        // 36 tiles of r = 64 over 8 warps
-inline size_t gram_mma_smem_bytes(int max_r) { return (size_t)((max_r + 7) & ~7) * kGramPitch * sizeof(float); }
+inline size_t gram_smem_bytes(int max_r) { return (size_t)((max_r + 7) & ~7) * kGramPitch * sizeof(float); }
 __device__ __forceinline__ void dmma_m8n8k4(double& c0, double& c1, double a, double b) {
   asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
                : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
-__global__ void __launch_bounds__(256) reduce_gram_mma_kernel(const DevLayer* __restrict__ layers, int l0, int y_reduced,
-                                                              int after_fused) {
+__global__ void __launch_bounds__(256) reduce_gram_kernel(const DevLayer* __restrict__ layers, int l0, int y_reduced,
+                                                          int after_fused) {
   const DevLayer& L = layers[l0 + blockIdx.y];
   const int nparts = y_parts(L, after_fused);
   const int ngroups = (L.gchunks + kGramGroup - 1) / kGramGroup;
@@ -431,6 +333,32 @@ __global__ void __launch_bounds__(kCholThreads) chol_kernel(const DevLayer* __re
   for (int a = 0; a < kCholOwn; ++a)
 #pragma unroll
     for (int c = 0; c < kCholOwn; ++c) sij[a][c] = 0.0;
+  if (r <= 32) {
+    // at most 2 x 2 elements per thread: four partial matrices are fetched at a time instead (added in chunk order)
+    for (int g0 = 0; g0 < ngroups; g0 += 4) {
+      double v[4][2][2];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const double* G = L.Gpart + (long long)min(g0 + u, ngroups - 1) * r * r;
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const int i = ti + 16 * a, j = tj + 16 * c;
+            v[u][a][c] = G[(i < r && j < r && j >= i) ? i * r + j : 0];
+          }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const int i = ti + 16 * a, j = tj + 16 * c;
+            sij[a][c] += (g0 + u < ngroups && i < r && j < r && j >= i) ? v[u][a][c] : 0.0;
+          }
+    }
+  } else
   for (int g = 0; g < ngroups; ++g) {
     const double* G = L.Gpart + (long long)g * r * r;
     double v[kCholOwn][kCholOwn];
@@ -747,10 +675,7 @@ cudaError_t launch_sum_slabs(const ExtractWave& w, cudaStream_t s) {
 cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStream_t s) {
   const int nl = w.l1 - w.l0;
   const dim3 gram_grid((w.max_gchunks + kGramGroup - 1) / kGramGroup, nl);
-  if (w.max_r > kGramMmaMinRank)      // the FP64 tensor-core form pays from a few 8 x 8 tiles per warp on
-    reduce_gram_mma_kernel<<<gram_grid, 256, gram_mma_smem_bytes(w.max_r), s>>>(w.d_layers, w.l0, w.y_reduced, w.after_fused);
-  else
-    reduce_gram_kernel<<<gram_grid, 256, gram_smem_bytes_upto(w.max_r), s>>>(w.d_layers, w.l0, w.y_reduced, w.after_fused);
+  reduce_gram_kernel<<<gram_grid, 256, gram_smem_bytes(w.max_r), s>>>(w.d_layers, w.l0, w.y_reduced, w.after_fused);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t chol_bytes = chol_smem_bytes(w.max_r);
@@ -761,7 +686,7 @@ cudaError_t launch_panel_qr(const ExtractWave& w, DevStatus* d_status, cudaStrea
   chol_kernel<<<nl, kCholThreads, chol_bytes, s>>>(w.d_layers, w.l0, d_status);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (w.max_r > kGramMmaMinRank) {
+  if (w.max_r > kApplyMmaMinRank) {   // below that the thread-per-column form is faster (5.3 against 3.5 ms per 168 launches at r = 16)
     const size_t bytes = apply_mma_smem_bytes(w.max_r);
     if (bytes > 48 * 1024) {
       e = cudaFuncSetAttribute(apply_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_mma_smem_bytes(AGZO_MAX_RANK));
