@@ -61,6 +61,7 @@ struct PlanOpts {
   bool share_inputs;     // consecutive layers with the same X are served by one sweep
   int extract_regions;   // 1: waves run one after another; 2: alternate waves use two scratch regions
                          // and two helper streams, so one wave's small kernels overlap the other's sweeps
+  const FusedCaps* fused_caps;   // what the device holds of the fused kernel; null when sizing without a device
 };
 
 }  // namespace
@@ -346,7 +347,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   };
   auto runs_fused = [&](const agzo_layer& a) {
     return opts.extract_fused && extract_path != 1 && extract_path != 3 && tc_available && tc_eligible(a) &&
-           fused_eligible(a, opts.extract_fused == 2) && (opts.extract_fused == 2 || !shares_input((int)(&a - L)));
+           fused_eligible(opts.fused_caps, a, opts.extract_fused == 2) && (opts.extract_fused == 2 || !shares_input((int)(&a - L)));
   };
   long long column_blocks = 0;
   for (int k = 0; k < n; ++k)
@@ -355,7 +356,7 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
   const bool long_slabs_any = column_blocks >= kLongSlabColumnBlocks;
   auto long_slabs_for = [&](const agzo_layer&) { return long_slabs_any; };
   auto y_parts_min = [&](const agzo_layer& a) {
-    return runs_fused(a) ? fused_parts_bound(a, fused_cluster_size(a, opts.extract_fused == 2)) : 0;
+    return runs_fused(a) ? fused_parts_bound(a, fused_cluster_size(opts.fused_caps, a, opts.extract_fused == 2)) : 0;
   };
   int i = 0;
   while (i < n) {
@@ -430,8 +431,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
             D.grp_NB = g == 0 ? rows : 0;
             D.tmaps = ws + maps_offset(n) + (size_t)(j + g) * kMapBytes;
             // the power steps of this layer run fused (X read once per step) where its shape allows
-            D.fz_C = runs_fused(a) ? fused_cluster_size(a, opts.extract_fused == 2) : 0;
-            D.fz_slice = fused_slice_cols(a, opts.extract_fused == 2);
+            D.fz_C = runs_fused(a) ? fused_cluster_size(opts.fused_caps, a, opts.extract_fused == 2) : 0;
+            D.fz_slice = fused_slice_cols(opts.fused_caps, a, opts.extract_fused == 2);
           }
         }
       }
@@ -463,7 +464,8 @@ agzo_status build_plan(const agzo_layer* L, int n, char* ws, size_t ws_bytes, co
       if (opts.extract_fused != 2 && xbytes <= kL2ResidentWaveBytes)
         for (int k = i; k < j; ++k) plan->dev[k].fz_C = 0;
       // the fused kernel's launches of this wave, one per cluster size: who works on which tiles
-      for (int C = 1; C <= 16; ++C) fused_plan_shares(plan->dev.data(), i, j, C);
+      if (opts.fused_caps)
+        for (int C = 1; C <= 16; ++C) fused_plan_shares(*opts.fused_caps, plan->dev.data(), i, j, C);
     }
     plan->wave_end.push_back(j);
     plan->wave_region.push_back(region);
@@ -502,7 +504,8 @@ agzo_status prepare(agzo_ctx* c, const agzo_layer* L, int n, cudaStream_t s) {
   Plan plan;
   PlanOpts opts{c->wave_bytes, c->extract_path, c->rmw_path, c->rmw_tc_min_rank, c->rmw_tc_panels, c->rmw_stage_r,
                 c->tc.available, c->extract_fused, c->share_inputs != 0,
-                c->allreduce ? 1 : c->extract_streams};   // the ranks' sums run in wave order on the caller's stream
+                c->allreduce ? 1 : c->extract_streams,    // the ranks' sums run in wave order on the caller's stream
+                &c->tc.fused};
   agzo_status st = build_plan(L, n, c->ws, c->ws_bytes, opts, &plan, nullptr);
   if (st == AGZO_ERR_WORKSPACE && opts.extract_regions == 2) {   // a workspace sized for one region
     opts.extract_regions = 1;
@@ -612,13 +615,13 @@ agzo_status agzo_workspace_bytes(const agzo_layer* h_layers, int n, size_t* h_by
   // the CUDA-core kernels, whose slabs are shaped differently)
   Plan plan;
   size_t scratch = 0, scratch_cc = 0;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 0, false, 2}, &plan, &scratch);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 0, false, 2, nullptr}, &plan, &scratch);
   if (st != AGZO_OK) return st;
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, 0, false, 2}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 1, 1, 0, 1, 1, false, 0, false, 2, nullptr}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   // ... and for the fused power step, whose layers keep room for one partial sum of Y per share of a launch
-  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 2, false, 2}, &plan, &scratch_cc);
+  st = build_plan(h_layers, n, nullptr, 0, PlanOpts{kDefaultWaveBytes, 0, 0, 3, 0, 0, true, 2, false, 2, nullptr}, &plan, &scratch_cc);
   if (st != AGZO_OK) return st;
   if (scratch_cc > scratch) scratch = scratch_cc;
   *h_bytes = kHeaderBytes + table_bytes(n) + scratch + kAlign;
@@ -797,7 +800,7 @@ agzo_status agzo_query_cluster_capacity(agzo_ctx* ctx, int32_t* h_clusters) {
   agzo_status st = check_ctx(ctx);
   if (st != AGZO_OK) return st;
   if (!h_clusters) return AGZO_ERR_INVALID_ARG;
-  for (int C = 0; C <= 16; ++C) h_clusters[C] = ctx->tc.available ? fused_resident_clusters(C) : 0;
+  for (int C = 0; C <= 16; ++C) h_clusters[C] = ctx->tc.available ? fused_resident_clusters(ctx->tc.fused, C) : 0;
   return AGZO_OK;
 }
 
@@ -913,7 +916,7 @@ agzo_status agzo_extract_subspace(agzo_ctx* ctx, const agzo_layer* h_layers, int
         for (int C = 1; C <= 16; ++C) {
           if (!(fz_classes & (1u << C))) continue;
           Timed t(ctx, AGZO_KC_FUSED_POWER, ws);
-          cudaError_t e = launch_fused_power_step(w, P.dev.data(), C, dst, ws);
+          cudaError_t e = launch_fused_power_step(ctx->tc.fused, w, P.dev.data(), C, dst, ws);
           if (e != cudaSuccess) return e;
         }
         return cudaSuccess;

@@ -507,11 +507,6 @@ fused_power_step_kernel(const DevLayer* __restrict__ layers, int l0, int l1, int
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, tmem_cols); }
 }
 
-// Clusters of this kernel that can be resident at once, per cluster size; filled by fused_init (a cluster
-// has to fit into one GPC, so sizes that do not divide a GPC's SMs leave part of the device idle).
-int g_max_clusters[2][kMaxCluster + 1] = {};   // [narrow / wide instantiation][cluster size]
-int g_sm_count = 0;                         // 0 until fused_init has run
-
 using FzKernel = void (*)(const DevLayer*, int, int, int, int, int, DevStatus*);
 FzKernel fz_kernel(bool wide, bool small) {
   return wide ? (small ? fused_power_step_kernel<true, true> : fused_power_step_kernel<true, false>)
@@ -548,7 +543,7 @@ cudaError_t fz_max_clusters(bool wide, int C, int sm_count, int* n) {
 // of the unfused kernels, which are faster then; 0 when neither width qualifies.  Before fused_init has
 // run (sizing a workspace without a device) the shape alone decides; with any_size the 70 % rule is
 // dropped (every cluster size that the device can launch at all).
-int fused_slice_cols(const agzo_layer& a, bool any_size) {
+int fused_slice_cols(const FusedCaps* caps, const agzo_layer& a, bool any_size) {
   const int NP = (a.r + 7) / 8 * 8;
   int best = 0;
   double best_share = -1.0;
@@ -558,10 +553,10 @@ int fused_slice_cols(const agzo_layer& a, bool any_size) {
     if (C * ((kGroups + C - 1) / C) * 8 * NP > (NP <= 8 ? FzCfg<false, true>::rs_floats : FzCfg<false, false>::rs_floats))
       continue;
     double share = 0.0;
-    if (g_sm_count) {
-      const int resident = g_max_clusters[slice > kSliceCols || C > 8][C];
+    if (caps && caps->sm_count) {
+      const int resident = caps->clusters[slice > kSliceCols || C > 8][C];
       if (resident <= 0) continue;
-      share = (double)a.d_in / slice * resident / g_sm_count;
+      share = (double)a.d_in / slice * resident / caps->sm_count;
       if (!any_size && share < 0.7) continue;
     }
     if (share > best_share) { best = slice; best_share = share; }
@@ -569,16 +564,16 @@ int fused_slice_cols(const agzo_layer& a, bool any_size) {
   return best;
 }
 
-int fused_cluster_size(const agzo_layer& a, bool any_size) {
-  const int slice = fused_slice_cols(a, any_size);
+int fused_cluster_size(const FusedCaps* caps, const agzo_layer& a, bool any_size) {
+  const int slice = fused_slice_cols(caps, a, any_size);
   return slice ? (a.d_in + slice - 1) / slice : 0;
 }
 
-bool fused_eligible(const agzo_layer& a, bool any_size) {
-  return tc_eligible(a) && a.r <= 16 && a.m >= kTT && fused_slice_cols(a, any_size) != 0;
+bool fused_eligible(const FusedCaps* caps, const agzo_layer& a, bool any_size) {
+  return tc_eligible(a) && a.r <= 16 && a.m >= kTT && fused_slice_cols(caps, a, any_size) != 0;
 }
 
-cudaError_t fused_init(int sm_count) {
+cudaError_t fused_init(int sm_count, FusedCaps* caps) {
   bool big = true;
   for (int wide = 0; wide < 2; ++wide)
     for (int small = 0; small < 2; ++small) {
@@ -593,17 +588,17 @@ cudaError_t fused_init(int sm_count) {
   for (int C = 1; C <= kMaxCluster; ++C) {
     int n = 0;
     if (C > 8 || fz_max_clusters(false, C, sm_count, &n) != cudaSuccess) n = 0;
-    g_max_clusters[0][C] = n;
+    caps->clusters[0][C] = n;
     n = 0;
     if ((C > 8 && !big) || fz_max_clusters(true, C, sm_count, &n) != cudaSuccess) n = 0;
-    g_max_clusters[1][C] = n;
+    caps->clusters[1][C] = n;
   }
   cudaGetLastError();
-  g_sm_count = sm_count;
+  caps->sm_count = sm_count;
   return cudaSuccess;
 }
 
-int fused_resident_clusters(int C) { return C >= 1 && C <= kMaxCluster ? g_max_clusters[C > 8][C] : 0; }
+int fused_resident_clusters(const FusedCaps& caps, int C) { return C >= 1 && C <= kMaxCluster ? caps.clusters[C > 8][C] : 0; }
 
 // The partial sums of Y that a fused power step can leave for a layer, at most: one per share that meets it.
 int fused_parts_bound(const agzo_layer& a, int C) {
@@ -633,7 +628,7 @@ int fused_split(const int* tiles, int n, int clusters, int* tile0, int* first, i
 int fused_share_begin(int k, int base, int rem) { return fz_share_begin(k, base, rem); }
 
 // Cuts the tiles of the layers of [l0, l1) with cluster size C into shares: fills fz_tile0, fz_first and fz_parts.
-void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
+void fused_plan_shares(const FusedCaps& caps, DevLayer* dev, int l0, int l1, int C) {
   std::vector<int> idx, tiles;
   bool wide = C > 8;
   for (int i = l0; i < l1; ++i)
@@ -646,7 +641,7 @@ void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
   const int n = (int)idx.size();
   std::vector<int> tile0(n), first(n), parts(n);
   int base = 0, rem = 0;
-  fused_split(tiles.data(), n, g_max_clusters[wide][C], tile0.data(), first.data(), parts.data(), &base, &rem);
+  fused_split(tiles.data(), n, caps.clusters[wide][C], tile0.data(), first.data(), parts.data(), &base, &rem);
   for (int k = 0; k < n; ++k) {
     dev[idx[k]].fz_tile0 = tile0[k];
     dev[idx[k]].fz_first = first[k];
@@ -655,8 +650,8 @@ void fused_plan_shares(DevLayer* dev, int l0, int l1, int C) {
 }
 
 // One fused power step for the layers of the wave whose cluster size is C.
-cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
-                                    cudaStream_t s) {
+cudaError_t launch_fused_power_step(const FusedCaps& caps, const ExtractWave& w, const DevLayer* h_dev, int C,
+                                    DevStatus* d_status, cudaStream_t s) {
   int total = 0;
   bool wide = C > 8, small = true;
   for (int i = w.l0; i < w.l1; ++i)
@@ -666,7 +661,7 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
       if (h_dev[i].NB > 16) small = false;
     }
   if (total == 0) return cudaSuccess;
-  if (C < 1 || C > kMaxCluster || g_max_clusters[wide][C] <= 0) return cudaErrorInvalidConfiguration;   // the planner picks no such size
+  if (C < 1 || C > kMaxCluster || caps.clusters[wide][C] <= 0) return cudaErrorInvalidConfiguration;   // the planner picks no such size
   cudaLaunchConfig_t cfg{};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -679,7 +674,7 @@ cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   // persistent clusters, never more than can be resident at once; the same count as fused_plan_shares used
-  const int nclusters = total < g_max_clusters[wide][C] ? total : g_max_clusters[wide][C];
+  const int nclusters = total < caps.clusters[wide][C] ? total : caps.clusters[wide][C];
   cfg.gridDim = dim3((unsigned)(nclusters * C));
   const DevLayer* layers = w.d_layers;
   int l0 = w.l0, l1 = w.l1;

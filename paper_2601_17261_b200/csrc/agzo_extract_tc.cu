@@ -418,7 +418,7 @@ cudaError_t tc_init(TcState* st, int device) {
     if (e == cudaSuccess) {
       int sms = 0;
       e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-      if (e == cudaSuccess) e = fused_init(sms);
+      if (e == cudaSuccess) e = fused_init(sms, &st->fused);
     }
     if (e != cudaSuccess) { cudaGetLastError(); st->available = false; }
   }

@@ -5,10 +5,19 @@
 
 namespace agzo {
 
+// What the context's device holds of the fused power-step kernel: thread-block clusters resident at once,
+// per instantiation (narrow / wide) and cluster size.  A cluster lives inside one GPC, so the counts differ
+// from chip to chip; they are asked once per context and everything that depends on them (which layers run
+// fused, how a launch's tiles are shared out, the launch's grid) reads this one copy.
+struct FusedCaps {
+  int sm_count = 0;            // 0: not asked yet (sizing a workspace without a device): shapes alone decide
+  int clusters[2][17] = {};
+};
 struct TcState {
   void* encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
   int device = -1;
   bool available = false;
+  FusedCaps fused;
 };
 
 cudaError_t tc_init(TcState* st, int device);
@@ -56,17 +65,17 @@ cudaError_t tc_x_q(const TcState& st, const ExtractWave& w, const DevLayer* h_de
 
 // ---- fused power step (agzo_extract_fused.cu): Y = X^T (X Q) in one pass over X
 // any_size: also cluster sizes that leave more than 30 % of the SMs idle
-bool fused_eligible(const agzo_layer& a, bool any_size);
-int fused_cluster_size(const agzo_layer& a, bool any_size);
-int fused_slice_cols(const agzo_layer& a, bool any_size);   // columns of X per CTA of the cluster, 0 = not eligible
+bool fused_eligible(const FusedCaps* caps, const agzo_layer& a, bool any_size);
+int fused_cluster_size(const FusedCaps* caps, const agzo_layer& a, bool any_size);
+int fused_slice_cols(const FusedCaps* caps, const agzo_layer& a, bool any_size);   // columns of X per CTA of the cluster, 0 = not eligible
 int fused_parts_bound(const agzo_layer& a, int C);              // partial sums of Y a power step can leave, at most
-void fused_plan_shares(DevLayer* dev, int l0, int l1, int C);   // fills fz_tile0 / fz_parts of a wave's layers of size C
-int fused_resident_clusters(int C);                             // clusters of C CTAs the device holds at once (after fused_init)
+void fused_plan_shares(const FusedCaps& caps, DevLayer* dev, int l0, int l1, int C);   // fills fz_tile0 / fz_first / fz_parts of a wave's layers of size C
+int fused_resident_clusters(const FusedCaps& caps, int C);      // clusters of C CTAs the device holds at once
 // the split on plain arrays and the first tile of share k (host; the kernel walks the same shares)
 int fused_split(const int* tiles, int n, int clusters, int* tile0, int* first, int* parts, int* base, int* rem);
 int fused_share_begin(int k, int base, int rem);
-cudaError_t fused_init(int sm_count);          // asks the device which cluster sizes fit; eligibility follows it
-cudaError_t launch_fused_power_step(const ExtractWave& w, const DevLayer* h_dev, int C, DevStatus* d_status,
-                                    cudaStream_t s);
+cudaError_t fused_init(int sm_count, FusedCaps* caps);   // asks the current device which cluster sizes fit
+cudaError_t launch_fused_power_step(const FusedCaps& caps, const ExtractWave& w, const DevLayer* h_dev, int C,
+                                    DevStatus* d_status, cudaStream_t s);
 
 }  // namespace agzo
