@@ -582,6 +582,27 @@ def test_extract_rank_deficient_panel_is_reported():
     assert projector_distance(Vg[:2], Vo[:2]) <= 1e-3
 
 
+@pytest.mark.parametrize("r,p", [(20, 13), (40, 17), (64, 33), (64, 1), (17, 16)])
+def test_extract_low_rank_input_across_the_register_tiles_of_the_factorisation(r, p):
+    """X of exact rank p < r: the factorisation meets its first dependent column at index p, which for
+    these sizes lies in every position of the 16 x 16 thread arrangement that owns the matrix (first,
+    second and third block of rows, a block boundary).  The dependent columns come out zero and flagged on
+    both sides, the others span the same space."""
+    rng = np.random.default_rng(r * 100 + p)
+    m, d_in = 512, 256
+    X = sum(np.outer(rng.standard_normal(m), rng.standard_normal(d_in)) for _ in range(p)).astype(np.float32)
+    Vg, st = _run_extract(X, r, 2, seed=3, layer_id=0, path=1, x_bf16=False)
+    assert st == B.AGZO_WARN_RANK_DEFICIENT
+    Vo, info = O.extract_subspace(X, r, 2, 3, 0, return_info=True)
+    assert info["deficient"]
+    live_g, live_o = np.abs(Vg).sum(1) > 0, np.abs(Vo).sum(1) > 0
+    assert live_g.sum() == live_o.sum() == p
+    assert np.array_equal(live_g, live_o)
+    Vl = Vg[live_g].astype(np.float64)
+    assert np.abs(Vl @ Vl.T - np.eye(p)).max() <= 1e-5
+    assert projector_distance(Vg[live_g], Vo[live_o]) <= 1e-3
+
+
 def test_empty_layer_list_and_argument_errors():
     V = torch.zeros(4, 64, device=DEV)
     W = torch.zeros(32, 64, device=DEV, dtype=torch.bfloat16)
